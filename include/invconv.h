@@ -1,0 +1,166 @@
+/*
+ * invconv.h -- C ABI of the B200 (sm_100a) library for the inverse of a masked,
+ * top-left-padded k x k multi-channel convolution and its backpropagation
+ * (Nagar & Varma, "Parallel Backpropagation for Inverse of a Convolution with
+ * Application to Normalizing Flows").
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - Unless a parameter is named *_host, every pointer is a DEVICE pointer to
+ *    contiguous fp32.  Activations x, y, grad_x, grad_y are [B][C][H][W];
+ *    kernels w, grad_w are [C_out][C_in][k][k].
+ *  - The kernel entry that multiplies pixel (h-dh, w-dw) in output pixel (h, w)
+ *    is w[co][ci][k-1-dh][k-1-dw], 0 <= dh, dw < k (Eq. 1; Algorithm 1's index
+ *    K[c, k_c, k_H-k_h-1, k_W-k_w-1]).  Pixels with a negative coordinate are
+ *    the zero padding on the top and left (Section 3).
+ *  - The bottom-right entry w[:, :, k-1, k-1] multiplies the output pixel
+ *    itself.  It is masked to ci <= co; its channel diagonal must be non-zero
+ *    (the paper fixes it to 1).  Values stored at ci > co on that tap are never
+ *    read.  A zero diagonal yields inf/nan, as in the paper where invertibility
+ *    is assumed.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *    stream).  Calls only enqueue work on `stream`: they never synchronise and
+ *    never free or keep caller memory.  The library is re-entrant; calls that
+ *    share a workspace must be ordered on one stream.
+ *  - Ownership: the caller owns every buffer.  Outputs are overwritten, never
+ *    accumulated into.  Inputs and outputs must not alias.
+ *  - Return value: an invconv_status (0 = success).  Nothing throws or aborts.
+ *    Pointers need no particular alignment: unaligned buffers take scalar
+ *    loads.
+ *  - Limits: 1 <= k <= INVCONV_MAX_K, 1 <= C <= INVCONV_MAX_C, B, H, W >= 1,
+ *    B*C*H*W < 2^31.  B == 0 is a successful no-op (grad_w is still zeroed).
+ */
+#ifndef INVCONV_H_
+#define INVCONV_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define INVCONV_MAX_K 11   /* largest kernel in the paper's ablation (Supplementary, kernel-size table) */
+#define INVCONV_MAX_C 128
+
+enum invconv_status {
+    INVCONV_OK = 0,
+    INVCONV_BAD_ARG = 1,          /* NULL pointer, non-positive size, aliasing in == out */
+    INVCONV_UNSUPPORTED = 2,      /* k or C beyond the compiled limits, tensor too large */
+    INVCONV_CUDA_ERROR = 3,       /* a launch or runtime call failed (cudaGetLastError) */
+    INVCONV_TIMEOUT = 4,          /* a bounded device-side wait gave up (see invconv_get_status) */
+    INVCONV_WORKSPACE_TOO_SMALL = 5
+};
+
+/* Which kernel family serves a call.  AUTO picks by shape; the others force a
+ * family (tests and measurements); a family that cannot serve the shape
+ * returns INVCONV_UNSUPPORTED. */
+enum invconv_path {
+    INVCONV_PATH_AUTO = 0,
+    INVCONV_PATH_GENERIC = 1,     /* one CTA per image, operands in global memory, any shape */
+    INVCONV_PATH_WARP = 2,        /* warp-shuffle wavefront, image resident in shared memory, small C */
+    INVCONV_PATH_TEAM = 3         /* CTA / cluster per image, register-tiled channel contraction, wide C */
+};
+
+/* x = f^{-1}(y): the inverse of the masked convolution, by wavefront
+ * substitution over the H+W-1 anti-diagonals (Section 3, Eq. 1 solved for
+ * x_q; Supplementary "Input Padding and Kernel Masking").
+ *   y [B,C,H,W] in, w [C,C,k,k] in, x [B,C,H,W] out.
+ * Uses stream-ordered scratch from the device's default memory pool when the
+ * shape needs a workspace (see invconv_workspace_bytes); use the _ws form to
+ * supply the scratch yourself. */
+int invconv_forward(const float* y, const float* w, float* x,
+                    int B, int C, int H, int W, int k, void* stream);
+
+/* Backpropagation through x = f^{-1}(y) (Section 3.1-3.3, Theorems 1 and 2,
+ * Algorithm 1's schedule):
+ *   grad_y = M^{-T} grad_x       reverse wavefront from the bottom-right corner,
+ *   grad_w[co][ci][k-1-dh][k-1-dw] = -sum_{n,h,w} grad_y[n,co,h,w] * x[n,ci,h-dh,w-dw],
+ *                                   summed over the batch; 0 outside the mask.
+ *   grad_x [B,C,H,W] in, x [B,C,H,W] in (the saved forward output), w in,
+ *   grad_y [B,C,H,W] out, grad_w [C,C,k,k] out.  grad_w may be NULL (skip it);
+ *   grad_y must be non-NULL (grad_w is computed from it). */
+int invconv_backward(const float* grad_x, const float* x, const float* w,
+                     float* grad_y, float* grad_w,
+                     int B, int C, int H, int W, int k, void* stream);
+
+/* y = f(x): the masked convolution itself, the sampling direction
+ * (Eq. 1; Section 4.3).  x in, w in, y out. */
+int masked_conv_forward(const float* x, const float* w, float* y,
+                        int B, int C, int H, int W, int k, void* stream);
+
+/* logdet[0] = H*W*sum_c log|w[c][c][k-1][k-1]| = log|det df/dx| (Section 4:
+ * triangular Jacobian; a unit diagonal gives 0).  Accumulated in double on the
+ * device and rounded once to fp32.  The inverse layer's log-det is its
+ * negative.  logdet points to ONE device float. */
+int invconv_logdet(const float* w, float* logdet, int C, int H, int W, int k, void* stream);
+
+/* Scratch bytes a forward or backward call of this shape needs (0 if none).
+ * Same value for both directions. */
+size_t invconv_workspace_bytes(int B, int C, int H, int W, int k);
+
+/* As invconv_forward / invconv_backward, but with caller-owned device scratch
+ * of at least invconv_workspace_bytes(...) bytes, 256-byte aligned.  These
+ * forms allocate nothing.  The first INVCONV_WS_CONTROL_BYTES bytes are
+ * control words: zero them once after allocating the workspace (cudaMemset);
+ * every call leaves them zero again.  Calls sharing a workspace must not
+ * overlap on the device. */
+#define INVCONV_WS_CONTROL_BYTES 256
+int invconv_forward_ws(const float* y, const float* w, float* x,
+                       int B, int C, int H, int W, int k,
+                       void* workspace, size_t workspace_bytes, void* stream);
+int invconv_backward_ws(const float* grad_x, const float* x, const float* w,
+                        float* grad_y, float* grad_w,
+                        int B, int C, int H, int W, int k,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* One whole layer step from HOST buffers: copies y, w, grad_x to the device,
+ * runs invconv_forward, invconv_backward and invconv_logdet there, and copies
+ * x, grad_y, grad_w and the log-det back -- all enqueued on `stream`, no
+ * synchronisation (use pinned host memory for truly asynchronous copies and
+ * synchronise the stream before reading the outputs).
+ *   *_host: host pointers (y, grad_x, x, grad_y: B*C*H*W floats; w, grad_w:
+ *   C*C*k*k floats; logdet: 1 float).
+ *   device_scratch: caller-owned device memory of at least
+ *   invconv_step_scratch_bytes(...) bytes, 256-byte aligned, zeroed once after
+ *   allocation; holds the device copies and the kernels' workspace. */
+size_t invconv_step_scratch_bytes(int B, int C, int H, int W, int k);
+int invconv_step_host(const float* y_host, const float* w_host, const float* grad_x_host,
+                      float* x_host, float* grad_y_host, float* grad_w_host, float* logdet_host,
+                      int B, int C, int H, int W, int k,
+                      void* device_scratch, size_t device_scratch_bytes, void* stream);
+
+/* Force a kernel family for subsequent calls from this process (default AUTO).
+ * Returns the previous setting. */
+int invconv_set_path(int path);
+
+/* The family AUTO would pick for this shape (an invconv_path value). */
+int invconv_path_for(int B, int C, int H, int W, int k);
+
+/* Synchronises `stream`, then reports and clears the device-side status word
+ * of the current device: INVCONV_OK, or INVCONV_TIMEOUT if a bounded wait
+ * inside a kernel gave up since the last query (its outputs are then invalid).
+ * Returns INVCONV_CUDA_ERROR if the synchronisation itself failed. */
+int invconv_get_status(void* stream, int* device_status_out);
+
+/* Measures, on the current device, the latency of one dependent wavefront step
+ * for a communication mechanism, with no other work on the chain:
+ *   mechanism 0: warp shuffle + one FMA (lane = image row);
+ *   mechanism 1: shared-memory store, block barrier, load, one FMA;
+ *   mechanism 2: store to a cluster peer's shared memory, cluster barrier, load, one FMA.
+ * Runs a chain of `steps` dependent steps in one CTA (cluster of 2 for 2) and
+ * writes the elapsed SM clock cycles to cycles_out[0] and the chain's final
+ * value to cycles_out[1] (device pointer to two 64-bit words).  Used for the
+ * critical-path bound of 2*(H+W-1) dependent steps (Section 3.3, complexity). */
+int invconv_probe_step_latency(int mechanism, int steps, unsigned long long* cycles_out, void* stream);
+
+/* Number of kernels this library has launched (or captured into a CUDA graph)
+ * from this process since it was loaded. */
+unsigned long long invconv_kernel_launch_count(void);
+
+const char* invconv_status_string(int status);
+int invconv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* INVCONV_H_ */

@@ -1,0 +1,33 @@
+// Shared declarations of the inverse-convolution kernels (device side).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "invconv.h"
+
+namespace invconv {
+
+// Problem geometry handed to every kernel.
+struct Geom {
+    int B, C, H, W, k;
+};
+
+// Device-side status word (one per device that loads the library).  Kernels
+// only ever raise it (atomicMax) when a bounded wait gives up.
+__device__ int g_device_status = 0;
+
+__device__ __forceinline__ void raise_status(int code) { atomicMax(&g_device_status, code); }
+
+// Index helpers.  Activations are [B][C][H][W]; kernels [C][C][k][k].
+__host__ __device__ __forceinline__ size_t act_index(int n, int c, int h, int w, int C, int H, int W) {
+    return (((size_t)n * C + c) * H + h) * W + w;
+}
+__host__ __device__ __forceinline__ int w_index(int co, int ci, int a, int b, int C, int k) {
+    return ((co * C + ci) * k + a) * k + b;
+}
+
+// Upper bound on polls of any device-side wait before it gives up.
+constexpr unsigned kMaxSpins = 1u << 22;
+
+}  // namespace invconv

@@ -1,0 +1,215 @@
+"""Parity of the CUDA library (through its C ABI) with the float64 oracle.
+
+Tolerances (normalised max error  max|a-b| / max|b|  per tensor; element-wise
+relative error is meaningless where outputs cross zero):
+    x, grad_y  <= 1e-4        grad_w <= 1e-3
+    log-det    |a-b| <= 1e-5 * max(|b|, H*W*1e-3)
+"""
+import numpy as np
+import pytest
+
+from conftest import nmax_err
+from paper_2410_14634_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+TOL_X = 1e-4
+TOL_GW = 1e-3
+
+PATHS = {"auto": 0, "generic": 1, "warp": 2, "team": 3}
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2410_14634_b200 import binding
+    binding.lib()
+    yield binding
+    binding.invconv_set_path(0)
+
+
+@pytest.fixture(scope="module")
+def oracle():
+    from oracle import api
+    return api
+
+
+def dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def run_or_skip(binding, fn, *args, **kw):
+    try:
+        return fn(*args, **kw)
+    except binding.InvConvError as e:
+        if e.status == binding.UNSUPPORTED:
+            pytest.skip("this kernel family does not serve the shape")
+        raise
+
+
+def check_all(binding, oracle, w, y, gx, path, tol_x=TOL_X, tol_gw=TOL_GW):
+    """Forward, backward (on the GPU's own x and on the oracle's x), f, log-det."""
+    import torch
+    Bn, C, H, W = y.shape
+    k = w.shape[2]
+    binding.invconv_set_path(PATHS[path])
+    try:
+        wd, yd, gxd = dev(w), dev(y), dev(gx)
+        x = run_or_skip(binding, binding.invconv_forward, yd, wd)
+        gy, gw = run_or_skip(binding, binding.invconv_backward, gxd, x, wd)
+        x_ref = oracle.invconv_forward(y, w)
+        gy_ref, gw_ref = oracle.invconv_backward(gx, x_ref, w)
+        # backward again from the oracle's x rounded to fp32 (separates forward from backward error)
+        gy2, gw2 = binding.invconv_backward(gxd, dev(x_ref.astype(np.float32)), wd)
+        yy = binding.masked_conv_forward(x, wd)
+        ld = binding.invconv_logdet(wd, H, W)
+        torch.cuda.synchronize()
+        assert binding.invconv_get_status() == 0
+    finally:
+        binding.invconv_set_path(0)
+    if Bn > 0:
+        assert nmax_err(x.cpu().numpy(), x_ref) <= tol_x
+        assert nmax_err(gy.cpu().numpy(), gy_ref) <= tol_x
+        assert nmax_err(gy2.cpu().numpy(), gy_ref) <= tol_x
+        assert nmax_err(yy.cpu().numpy(), y) <= tol_x                 # f(f^{-1}(y)) = y on the device
+    assert nmax_err(gw.cpu().numpy(), gw_ref) <= tol_gw
+    assert nmax_err(gw2.cpu().numpy(), gw_ref) <= tol_gw
+    ctr = gw.cpu().numpy()[:, :, k - 1, k - 1]
+    assert np.all(ctr[np.triu_indices(C, 1)] == 0.0)                  # outside the mask: exact zeros
+    ld_ref = oracle.logdet(w, H, W)
+    assert abs(float(ld.item()) - ld_ref) <= 1e-5 * max(abs(ld_ref), H * W * 1e-3)
+
+
+# ------------------------------------------------------------------ the ten benchmark shapes, full size
+
+@pytest.mark.parametrize("path", ["auto", "generic", "warp", "team"])
+@pytest.mark.parametrize("name", [s.name for s in workloads.SHAPES])
+def test_benchmark_shapes_full_size(B, oracle, name, path):
+    s, w, y, gx = workloads.make(name)
+    if path == "generic" and s.C * s.k * s.k > 1300:
+        pytest.skip("fallback kernel on the heaviest shapes is covered by the smaller cases")
+    check_all(B, oracle, w, y, gx, path)
+
+
+# ------------------------------------------------------------------ small, ragged and degenerate shapes
+
+EDGE = [  # (B, C, H, W, k)
+    (1, 1, 1, 1, 1), (2, 1, 1, 1, 3), (1, 2, 1, 5, 2), (1, 3, 6, 1, 3), (2, 2, 2, 2, 4),
+    (3, 1, 3, 3, 3), (2, 3, 5, 4, 3), (1, 2, 7, 9, 5), (2, 1, 13, 17, 2), (1, 3, 31, 29, 3),
+    (2, 1, 33, 30, 3), (1, 3, 35, 37, 5), (1, 4, 9, 11, 3), (1, 5, 6, 7, 3), (1, 7, 5, 5, 2),
+    (2, 12, 5, 7, 3), (1, 16, 9, 9, 3), (1, 33, 4, 6, 3), (1, 24, 8, 8, 5), (1, 1, 40, 70, 7),
+    (1, 2, 16, 16, 11), (1, 1, 65, 66, 3), (1, 3, 100, 20, 3), (5, 1, 28, 28, 3),
+]
+
+
+@pytest.mark.parametrize("path", ["auto", "generic", "warp", "team"])
+@pytest.mark.parametrize("shape", EDGE, ids=lambda s: "x".join(map(str, s)))
+def test_edge_shapes(B, oracle, shape, path):
+    Bn, C, H, W, k = shape
+    w, y, gx = workloads.make_custom(100 + sum(shape), Bn, C, H, W, k, sigma=0.05 / np.sqrt(C))
+    check_all(B, oracle, w, y, gx, path)
+
+
+@pytest.mark.parametrize("path", ["auto", "generic", "warp", "team"])
+def test_masked_out_kernel_entries_are_never_read(B, oracle, path):
+    for (Bn, C, H, W, k) in [(2, 3, 9, 8, 3), (1, 12, 6, 6, 3)]:
+        w, y, gx = workloads.make_custom(7, Bn, C, H, W, k, masked_fill=float("nan"))
+        check_all(B, oracle, w, y, gx, path)
+
+
+@pytest.mark.parametrize("path", ["auto", "generic", "warp", "team"])
+def test_paper_setting_unit_diagonal_one_channel(B, oracle, path):
+    """The paper's own assumption: one channel, bottom-right entry equal to 1; log-det is exactly 0."""
+    w, y, gx = workloads.make_custom(8, 3, 1, 12, 10, 3, diag_lo=1.0, diag_hi=1.0)
+    assert w[0, 0, 2, 2] == 1.0
+    check_all(B, oracle, w, y, gx, path)
+    assert float(B.invconv_logdet(dev(w), 12, 10).item()) == 0.0
+
+
+def test_empty_batch_is_a_no_op_and_zeroes_grad_w(B):
+    import torch
+    w = dev(workloads.make_custom(9, 1, 2, 4, 4, 3)[0])
+    y = torch.empty(0, 2, 4, 4, device="cuda")
+    x = B.invconv_forward(y, w)
+    gy, gw = B.invconv_backward(y, x, w)
+    torch.cuda.synchronize()
+    assert x.shape == y.shape and gy.shape == y.shape
+    assert torch.all(gw == 0)
+
+
+def test_results_are_bitwise_reproducible(B):
+    import torch
+    for name in ("pr1", "cifar_sq"):
+        s, w, y, gx = workloads.make(name)
+        wd, yd, gxd = dev(w), dev(y), dev(gx)
+        x1 = B.invconv_forward(yd, wd)
+        gy1, gw1 = B.invconv_backward(gxd, x1, wd)
+        x2 = B.invconv_forward(yd, wd)
+        gy2, gw2 = B.invconv_backward(gxd, x2, wd)
+        torch.cuda.synchronize()
+        assert torch.equal(x1, x2) and torch.equal(gy1, gy2) and torch.equal(gw1, gw2)
+
+
+def test_plain_entry_points_match_workspace_entry_points(B):
+    """invconv_forward / invconv_backward (library-managed scratch) against the _ws forms the binding uses."""
+    import torch
+    for name in ("pr1", "cifar_sq"):
+        s, w, y, gx = workloads.make(name)
+        wd, yd, gxd = dev(w), dev(y), dev(gx)
+        x_ws = B.invconv_forward(yd, wd)
+        gy_ws, gw_ws = B.invconv_backward(gxd, x_ws, wd)
+        x = torch.empty_like(yd); gy = torch.empty_like(yd); gw = torch.empty_like(wd)
+        L = B.lib()
+        st = torch.cuda.current_stream().cuda_stream
+        assert L.invconv_forward(yd.data_ptr(), wd.data_ptr(), x.data_ptr(), s.B, s.C, s.H, s.W, s.k, st) == 0
+        assert L.invconv_backward(gxd.data_ptr(), x.data_ptr(), wd.data_ptr(), gy.data_ptr(), gw.data_ptr(),
+                                  s.B, s.C, s.H, s.W, s.k, st) == 0
+        torch.cuda.synchronize()
+        assert torch.equal(x, x_ws) and torch.equal(gy, gy_ws) and torch.equal(gw, gw_ws)
+
+
+def test_grad_w_may_be_skipped(B):
+    import torch
+    s, w, y, gx = workloads.make("pr1")
+    wd, yd, gxd = dev(w), dev(y), dev(gx)
+    x = B.invconv_forward(yd, wd)
+    gy_a, _ = B.invconv_backward(gxd, x, wd)
+    gy_b, none = B.invconv_backward(gxd, x, wd, need_grad_w=False)
+    torch.cuda.synchronize()
+    assert none is None and torch.equal(gy_a, gy_b)
+
+
+def test_host_step_matches_oracle(B, oracle):
+    import torch
+    s, w, y, gx = workloads.make("pr1")
+    hs = B.HostStep(s.B, s.C, s.H, s.W, s.k)
+    hs.y.copy_(torch.from_numpy(y)); hs.w.copy_(torch.from_numpy(w)); hs.grad_x.copy_(torch.from_numpy(gx))
+    for _ in range(2):
+        hs.run()
+        torch.cuda.synchronize()
+        x_ref = oracle.invconv_forward(y, w)
+        gy_ref, gw_ref = oracle.invconv_backward(gx, x_ref, w)
+        assert nmax_err(hs.x.numpy(), x_ref) <= TOL_X
+        assert nmax_err(hs.grad_y.numpy(), gy_ref) <= TOL_X
+        assert nmax_err(hs.grad_w.numpy(), gw_ref) <= TOL_GW
+        ld_ref = oracle.logdet(w, s.H, s.W)
+        assert abs(float(hs.logdet.item()) - ld_ref) <= 1e-5 * max(abs(ld_ref), s.H * s.W * 1e-3)
+
+
+def test_bad_arguments_return_status_codes(B):
+    import torch
+    L = B.lib()
+    t = torch.zeros(64, device="cuda")
+    p = t.data_ptr()
+    assert L.invconv_forward(p, p, p, 1, 1, 4, 4, 3, None) == B.BAD_ARG            # x aliases y
+    assert L.invconv_forward(None, p, p, 1, 1, 4, 4, 3, None) == B.BAD_ARG
+    assert L.invconv_backward(p, p, p, None, None, 1, 1, 4, 4, 3, None) == B.BAD_ARG
+    assert L.invconv_forward(p, p, p, 1, 1, 4, 4, 12, None) == B.UNSUPPORTED
+    assert L.masked_conv_forward(p, p, p, 1, 1, 4, 4, 3, None) == B.BAD_ARG
+    assert B.invconv_get_status() == 0
+
+
+def test_step_latency_probes_run(B):
+    for mech in (0, 1, 2):
+        c = B.invconv_probe_step_latency(mech, 2048)
+        assert 1.0 < c < 5000.0
