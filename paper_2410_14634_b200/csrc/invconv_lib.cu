@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "generic_kernels.cuh"
 #include "probe_kernels.cuh"
+#include "warp_kernels.cuh"
 
 using namespace invconv;
 
@@ -43,9 +44,98 @@ int check_shape(int B, int C, int H, int W, int k)
     return INVCONV_OK;
 }
 
+constexpr size_t kMaxDynSmem = 226 * 1024;   // 227 KiB per CTA minus the kernels' static shared memory
+
+// ---------------------------------------------------------------- warp family
+#define INVCONV_WARP_CASES(X) \
+    X(1, 2) X(1, 3) X(1, 5) X(2, 2) X(2, 3) X(2, 5) X(3, 2) X(3, 3) X(3, 5) X(4, 2) X(4, 3) X(4, 5)
+
+struct WarpPlan {
+    bool ok = false;
+    int nb = 0, ipc = 0, grid = 0;
+    size_t smem = 0;
+};
+
+template <int C, int K>
+WarpPlan plan_warp_ck(int B, int H, int W, bool bwd)
+{
+    WarpPlan pl;
+    pl.nb = (H + 31) / 32;
+    if (pl.nb > 8) return pl;
+    int ipc = 4 / pl.nb;
+    if (ipc < 1) ipc = 1;
+    if (ipc > B) ipc = B > 0 ? B : 1;
+    while (ipc > 1 && warp_kernel_smem<C, K>(H, W, pl.nb, ipc, bwd) > kMaxDynSmem) --ipc;
+    pl.smem = warp_kernel_smem<C, K>(H, W, pl.nb, ipc, bwd);
+    if (pl.smem > kMaxDynSmem) return pl;
+    pl.ipc = ipc;
+    pl.grid = (B + ipc - 1) / ipc;
+    pl.ok = true;
+    return pl;
+}
+
+WarpPlan plan_warp(int B, int C, int H, int W, int k, bool bwd)
+{
+#define X(CC, KK) if (C == CC && k == KK) return plan_warp_ck<CC, KK>(B, H, W, bwd);
+    INVCONV_WARP_CASES(X)
+#undef X
+    return WarpPlan{};
+}
+
+template <typename Kern>
+int set_smem_limit(Kern kern, size_t smem)
+{
+    if (smem <= 48 * 1024) return INVCONV_OK;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        cudaGetLastError();
+        return INVCONV_CUDA_ERROR;
+    }
+    return INVCONV_OK;
+}
+
+template <int C, int K, bool BWD>
+int launch_warp_ck(const WarpPlan& pl, WarpParams prm, cudaStream_t st)
+{
+    auto kern = pl.nb > 1 ? warp_wavefront_kernel<C, K, BWD, true> : warp_wavefront_kernel<C, K, BWD, false>;
+    const int rc = set_smem_limit(kern, pl.smem);
+    if (rc) return rc;
+    kern<<<pl.grid, pl.nb * pl.ipc * 32, pl.smem, st>>>(prm);
+    return check_launch();
+}
+
+int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const float* xsaved, float* gw, Geom g,
+                void* ws, cudaStream_t st)
+{
+    const WarpPlan pl = plan_warp(g.B, g.C, g.H, g.W, g.k, bwd);
+    if (!pl.ok) return INVCONV_UNSUPPORTED;
+    WarpParams prm;
+    prm.rhs = rhs; prm.w = w; prm.out = out; prm.xsaved = xsaved; prm.grad_w = gw;
+    prm.counter = static_cast<unsigned*>(ws);
+    prm.partials = ws ? reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES) : nullptr;
+    prm.B = g.B; prm.H = g.H; prm.W = g.W; prm.nb = pl.nb; prm.ipc = pl.ipc;
+    const size_t chw = (size_t)g.C * g.H * g.W;
+    const bool aligned = ((reinterpret_cast<uintptr_t>(rhs) | reinterpret_cast<uintptr_t>(out) |
+                           reinterpret_cast<uintptr_t>(xsaved)) & 15) == 0;
+    prm.bulk = (aligned && chw % 4 == 0) ? 1 : 0;
+#define X(CC, KK)                                                                         \
+    if (g.C == CC && g.k == KK)                                                           \
+        return bwd ? launch_warp_ck<CC, KK, true>(pl, prm, st) : launch_warp_ck<CC, KK, false>(pl, prm, st);
+    INVCONV_WARP_CASES(X)
+#undef X
+    return INVCONV_UNSUPPORTED;
+}
+
+size_t warp_workspace_bytes(int B, int C, int H, int W, int k)
+{
+    const WarpPlan pl = plan_warp(B, C, H, W, k, true);
+    if (!pl.ok) return 0;
+    return INVCONV_WS_CONTROL_BYTES + sizeof(float) * (size_t)pl.grid * C * C * k * k;
+}
+
+// ---------------------------------------------------------------- dispatch
 int auto_path(int B, int C, int H, int W, int k)
 {
-    (void)B; (void)C; (void)H; (void)W; (void)k;
+    if (plan_warp(B > 0 ? B : 1, C, H, W, k, true).ok) return INVCONV_PATH_WARP;
     return INVCONV_PATH_GENERIC;
 }
 
@@ -57,19 +147,21 @@ int resolve_path(int B, int C, int H, int W, int k)
 
 size_t workspace_bytes_for(int path, int B, int C, int H, int W, int k)
 {
-    (void)path; (void)B; (void)C; (void)H; (void)W; (void)k;
+    if (path == INVCONV_PATH_WARP) return warp_workspace_bytes(B, C, H, W, k);
     return 0;
 }
 
 int launch_forward(int path, const float* y, const float* w, float* x, Geom g,
                    void* ws, size_t ws_bytes, cudaStream_t st)
 {
-    (void)ws; (void)ws_bytes;
+    (void)ws_bytes;
     if (g.B == 0) return INVCONV_OK;
     switch (path) {
     case INVCONV_PATH_GENERIC:
         generic_wavefront_kernel<false><<<g.B, 256, 0, st>>>(y, w, x, g);
         return check_launch();
+    case INVCONV_PATH_WARP:
+        return launch_warp(false, y, w, x, nullptr, nullptr, g, ws, st);
     default:
         return INVCONV_UNSUPPORTED;
     }
@@ -78,7 +170,7 @@ int launch_forward(int path, const float* y, const float* w, float* x, Geom g,
 int launch_backward(int path, const float* gx, const float* x, const float* w, float* gy, float* gw, Geom g,
                     void* ws, size_t ws_bytes, cudaStream_t st)
 {
-    (void)ws; (void)ws_bytes;
+    (void)ws_bytes;
     switch (path) {
     case INVCONV_PATH_GENERIC: {
         if (g.B > 0) {
@@ -92,6 +184,8 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
         }
         return INVCONV_OK;
     }
+    case INVCONV_PATH_WARP:
+        return launch_warp(true, gx, w, gy, x, gw, g, ws, st);
     default:
         return INVCONV_UNSUPPORTED;
     }
@@ -126,6 +220,7 @@ int invconv_forward_ws(const float* y, const float* w, float* x, int B, int C, i
 {
     const int rc = check_shape(B, C, H, W, k);
     if (rc) return rc;
+    if (B == 0) return w ? INVCONV_OK : INVCONV_BAD_ARG;
     if (!y || !w || !x || y == x) return INVCONV_BAD_ARG;
     const int path = resolve_path(B, C, H, W, k);
     const size_t need = workspace_bytes_for(path, B, C, H, W, k);
@@ -138,6 +233,14 @@ int invconv_backward_ws(const float* grad_x, const float* x, const float* w, flo
 {
     const int rc = check_shape(B, C, H, W, k);
     if (rc) return rc;
+    if (B == 0) {
+        if (!w) return INVCONV_BAD_ARG;
+        if (grad_w && cudaMemsetAsync(grad_w, 0, sizeof(float) * C * C * k * k, as_stream(stream)) != cudaSuccess) {
+            cudaGetLastError();
+            return INVCONV_CUDA_ERROR;
+        }
+        return INVCONV_OK;
+    }
     if (!grad_x || !x || !w || !grad_y || grad_x == grad_y || x == grad_y) return INVCONV_BAD_ARG;
     const int path = resolve_path(B, C, H, W, k);
     const size_t need = workspace_bytes_for(path, B, C, H, W, k);
@@ -150,8 +253,9 @@ int invconv_forward(const float* y, const float* w, float* x, int B, int C, int 
 {
     const int rc = check_shape(B, C, H, W, k);
     if (rc) return rc;
+    if (B > 0 && (!y || !w || !x || y == x)) return INVCONV_BAD_ARG;
     StreamScratch sc;
-    const size_t need = workspace_bytes_for(resolve_path(B, C, H, W, k), B, C, H, W, k);
+    const size_t need = B > 0 ? workspace_bytes_for(resolve_path(B, C, H, W, k), B, C, H, W, k) : 0;
     const int ra = sc.acquire(need, as_stream(stream));
     if (ra) return ra;
     return invconv_forward_ws(y, w, x, B, C, H, W, k, sc.p, need, stream);
@@ -162,8 +266,9 @@ int invconv_backward(const float* grad_x, const float* x, const float* w, float*
 {
     const int rc = check_shape(B, C, H, W, k);
     if (rc) return rc;
+    if (B > 0 && (!grad_x || !x || !w || !grad_y || grad_x == grad_y || x == grad_y)) return INVCONV_BAD_ARG;
     StreamScratch sc;
-    const size_t need = workspace_bytes_for(resolve_path(B, C, H, W, k), B, C, H, W, k);
+    const size_t need = B > 0 ? workspace_bytes_for(resolve_path(B, C, H, W, k), B, C, H, W, k) : 0;
     const int ra = sc.acquire(need, as_stream(stream));
     if (ra) return ra;
     return invconv_backward_ws(grad_x, x, w, grad_y, grad_w, B, C, H, W, k, sc.p, need, stream);
@@ -173,8 +278,8 @@ int masked_conv_forward(const float* x, const float* w, float* y, int B, int C, 
 {
     const int rc = check_shape(B, C, H, W, k);
     if (rc) return rc;
+    if (B == 0) return w ? INVCONV_OK : INVCONV_BAD_ARG;
     if (!x || !w || !y || x == y) return INVCONV_BAD_ARG;
-    if (B == 0) return INVCONV_OK;
     const long long total = (long long)B * C * H * W;
     const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
     generic_masked_conv_kernel<<<blocks, 256, 0, as_stream(stream)>>>(x, w, y, Geom{B, C, H, W, k}, total);

@@ -1,0 +1,540 @@
+// Warp-shuffle wavefront for few channels (C <= 4).
+//
+// One warp owns a block of 32 image rows: lane l solves row 32*j + l and, at
+// local step s, the pixel in column s - l, so a warp walks one anti-diagonal
+// per step (Section 3: pixels on one anti-diagonal are unordered and solved in
+// parallel; the diagonals follow one another).  The k-1 already-solved
+// neighbours in the lane's own row live in its registers; the rows above
+// arrive from the lanes above by one shuffle per row and channel, so a step
+// needs no barrier.  The whole image sits in shared memory, brought in by one
+// bulk (TMA) copy and solved in place, then written back by one bulk copy, so
+// every HBM access is a full contiguous transfer.
+//
+// Images taller than 32 rows use several warps: row block j starts a column as
+// soon as block j-1 has published it (a progress counter in shared memory,
+// polled every 8 steps with a bounded spin), i.e. the blocks run as a skewed
+// pipeline instead of a global lock-step.
+//
+// The channel solve of the centre tap is folded into the taps once per call:
+// with L = w[:, :, k-1, k-1] (lower triangular) the recurrence
+//     L x_p = y_p - sum_{delta != 0} W_delta x_{p-delta}
+// is solved as  x_p = L^-1 y_p - sum (L^-1 W_delta) x_{p-delta},
+// which is the paper's own unit-diagonal form (Section 3) for the transformed
+// kernel.  The transposed solve (grad_y, Theorem 1) is the same walk on the
+// image rotated by 180 degrees with  L^-T W_delta^T.
+//
+// grad_w (Theorem 2) is accumulated after the reverse wavefront from the two
+// images still resident in shared memory (grad_y and x): lane = column, rows
+// in order, a k x k window of x in registers; warp partials are combined per
+// CTA and the last CTA to finish sums the CTA partials in a fixed order.
+#pragma once
+
+#include "common.cuh"
+#include "tma.cuh"
+
+namespace invconv {
+
+struct WarpParams {
+    const float* rhs;      // y (forward) or grad_x (backward)
+    const float* w;        // [C][C][K][K]
+    float* out;            // x (forward) or grad_y (backward)
+    const float* xsaved;   // backward: the saved forward output x
+    float* grad_w;         // backward: may be nullptr
+    float* partials;       // backward: [gridDim.x][K*K*C*C] scratch
+    unsigned* counter;     // backward: one control word, zero on entry and on exit
+    int B, H, W;
+    int nb;                // row blocks (warps) per image
+    int ipc;               // images per CTA
+    int bulk;              // images are 16-byte aligned multiples of 16 bytes
+};
+
+template <int C> struct ColVec;
+template <> struct ColVec<1> { using type = float;  static constexpr int CP = 1; };
+template <> struct ColVec<2> { using type = float2; static constexpr int CP = 2; };
+template <> struct ColVec<3> { using type = float4; static constexpr int CP = 4; };
+template <> struct ColVec<4> { using type = float4; static constexpr int CP = 4; };
+
+template <int C, int K>
+struct WarpShape {
+    static constexpr int KK = K * K;
+    static constexpr int CP = ColVec<C>::CP;
+    static constexpr int NA = KK * C * C;           // kernel entries
+    static constexpr int NAP = KK * C * CP;         // padded copy in shared memory
+    static constexpr bool WREG = NA <= 144;         // transformed kernel held in registers
+    static constexpr int COB = (NA <= 100) ? C : 1; // output channels per grad_w pass
+};
+
+// Column a = 0..C-1 of the transformed kernel for (tap, input channel b).
+template <int C>
+__device__ __forceinline__ void load_col(const float* As, int idx, float (&col)[C])
+{
+    using V = typename ColVec<C>::type;
+    const V v = reinterpret_cast<const V*>(As)[idx];
+    if constexpr (C == 1) { col[0] = v; }
+    else if constexpr (C == 2) { col[0] = v.x; col[1] = v.y; }
+    else if constexpr (C == 3) { col[0] = v.x; col[1] = v.y; col[2] = v.z; }
+    else { col[0] = v.x; col[1] = v.y; col[2] = v.z; col[3] = v.w; }
+}
+
+// Transformed kernel into shared memory: As[(tap*C + b)*CP + a], tap = dh*K + dw,
+//   forward : tap 0 -> L^-1[a][b];          tap != 0 -> (L^-1 W_delta)[a][b]
+//   backward: tap 0 -> L^-1[b][a];          tap != 0 -> sum_m L^-1[m][a] w[b][m][delta]
+// where W_delta[co][ci] = w[co][ci][K-1-dh][K-1-dw].
+template <int C, int K, bool BWD>
+__device__ void build_transformed_kernel(const float* __restrict__ w, float* As)
+{
+    constexpr int KK = K * K, CP = ColVec<C>::CP;
+    constexpr int ctr = KK - 1;
+    float L[C][C], Li[C][C];
+#pragma unroll
+    for (int i = 0; i < C; ++i)
+#pragma unroll
+        for (int j = 0; j < C; ++j) {
+            L[i][j] = (j <= i) ? __ldg(w + (i * C + j) * KK + ctr) : 0.f;
+            Li[i][j] = 0.f;
+        }
+#pragma unroll
+    for (int j = 0; j < C; ++j) {
+        Li[j][j] = 1.0f / L[j][j];
+#pragma unroll
+        for (int i = j + 1; i < C; ++i) {
+            float s = 0.f;
+#pragma unroll
+            for (int m = j; m < i; ++m) s += L[i][m] * Li[m][j];
+            Li[i][j] = -s / L[i][i];
+        }
+    }
+    for (int e = threadIdx.x; e < KK * C * C; e += blockDim.x) {
+        const int a = e % C, b = (e / C) % C, tap = e / (C * C);
+        const int dh = tap / K, dw = tap % K;
+        const int t = (K - 1 - dh) * K + (K - 1 - dw);
+        float v = 0.f;
+        if (tap == 0) {
+#pragma unroll
+            for (int i = 0; i < C; ++i)
+#pragma unroll
+                for (int j = 0; j < C; ++j)
+                    if (i == (BWD ? b : a) && j == (BWD ? a : b)) v = Li[i][j];
+        } else {
+#pragma unroll
+            for (int m = 0; m < C; ++m) {
+                float li = 0.f;
+#pragma unroll
+                for (int i = 0; i < C; ++i)
+#pragma unroll
+                    for (int j = 0; j < C; ++j)
+                        if (i == (BWD ? m : a) && j == (BWD ? a : m)) li = Li[i][j];
+                const float wv = BWD ? __ldg(w + (b * C + m) * KK + t) : __ldg(w + (m * C + b) * KK + t);
+                v += li * wv;
+            }
+        }
+        As[(tap * C + b) * CP + a] = v;
+    }
+}
+
+// The wavefront over one block of up to 32 rows.  Logical pixel (lh, lw) of
+// channel c lives at img[c*HW + origin + sgn*(lh*W + lw)] (sgn = -1 walks the
+// rotated image of the transposed solve).  Returns false if a wait gave up.
+//
+// The step loop is unrolled by K-1 so that the sliding windows of solved
+// neighbours rotate through registers by renaming instead of moves: the value
+// produced at step s lives in slot s mod (K-1).  Lanes that have no row above
+// inside the block (lane <= d for the row d+1 above) get zeroed copies of the
+// taps that read those rows when the block is the image's first, so the
+// shuffle result feeds the FMA directly with no select on the dependent chain.
+template <int C, int K, bool MULTI>
+__device__ __forceinline__ bool wavefront_block(float* img, const float* As, int H, int W, int origin, int sgn,
+                                                int j, volatile int* progress, int lane)
+{
+    using S = WarpShape<C, K>;
+    constexpr int KM = K - 1;
+    const int HW = H * W;
+    const int rows = min(32, H - 32 * j);
+    const int nsteps = W + rows - 1;
+    const int nsteps_up = (nsteps + KM - 1) / KM * KM;
+    const int prod_steps = (W + 31 + KM - 1) / KM * KM;
+    const unsigned Wl = lane < rows ? (unsigned)W : 0u;     // active  <=>  (unsigned)lw < Wl
+    const bool first_block = !MULTI || j == 0;
+
+    float Ar[S::WREG ? S::NA : 1];
+    if constexpr (S::WREG) {
+#pragma unroll
+        for (int t = 0; t < S::KK * C; ++t) {
+            float col[C];
+            load_col<C>(As, t, col);
+            const int dh = t / (C * K);
+            const bool dead = first_block && dh >= 1 && lane < dh;   // the row dh above lies outside the image
+#pragma unroll
+            for (int a = 0; a < C; ++a) Ar[t * C + a] = dead ? 0.f : col[a];
+        }
+    }
+    float own[C][KM];          // slot (s mod KM) <- x[b][lh][lw] of step s
+    float up[KM][C][KM];       // slot (s mod KM) <- x[b][lh-1-d][lw] of step s
+#pragma unroll
+    for (int b = 0; b < C; ++b)
+#pragma unroll
+        for (int q = 0; q < KM; ++q) {
+            own[b][q] = 0.f;
+#pragma unroll
+            for (int d = 0; d < KM; ++d) up[d][b][q] = 0.f;
+        }
+    int p = origin + sgn * ((32 * j + lane) * W - lane);    // offset of (lh, lw) at step 0
+    float rnext[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) rnext[c] = (lane == 0 && Wl > 0) ? img[c * HW + p] : 0.f;
+
+    for (int s0 = 0; s0 < nsteps_up; s0 += KM) {
+        if constexpr (MULTI) {
+            if (j > 0 && (s0 & 7) == 0) {
+                const int need = min(s0 + 39, prod_steps);
+                unsigned spins = 0;
+                bool ok = true;
+                while (progress[j - 1] < need) {
+                    if (++spins > kMaxSpins) { ok = false; break; }
+                }
+                if (!__all_sync(0xffffffffu, ok)) return false;
+                __threadfence_block();
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < KM; ++u) {
+            const unsigned ulw = (unsigned)(s0 + u - lane);
+            const bool active = ulw < Wl;
+            float r[C];
+#pragma unroll
+            for (int c = 0; c < C; ++c) r[c] = rnext[c];
+            {
+                const bool act1 = (ulw + 1u) < Wl;
+#pragma unroll
+                for (int c = 0; c < C; ++c) rnext[c] = act1 ? img[c * HW + p + sgn] : 0.f;
+            }
+            // newest column of the rows above: by shuffle inside the block, from shared memory across blocks
+            float nu[KM][C];
+#pragma unroll
+            for (int d = 0; d < KM; ++d)
+#pragma unroll
+                for (int b = 0; b < C; ++b) {
+                    float v = __shfl_up_sync(0xffffffffu, own[b][(u - 1 - d + 2 * KM) % KM], d + 1);
+                    if constexpr (MULTI) {
+                        if (lane <= d) {
+                            v = 0.f;
+                            if (j > 0 && active) v = img[b * HW + p - sgn * (d + 1) * W];
+                        }
+                    } else if constexpr (!S::WREG) {
+                        if (lane <= d) v = 0.f;
+                    }
+                    nu[d][b] = v;
+                }
+            // everything that does not depend on the previous step's result
+            float acc[C], acc2[C];
+#pragma unroll
+            for (int a = 0; a < C; ++a) { acc[a] = 0.f; acc2[a] = 0.f; }
+#pragma unroll
+            for (int b = 0; b < C; ++b) {
+                float col[C];
+                if constexpr (S::WREG) {
+#pragma unroll
+                    for (int a = 0; a < C; ++a) col[a] = Ar[b * C + a];
+                } else load_col<C>(As, b, col);
+#pragma unroll
+                for (int a = 0; a < C; ++a) acc[a] = fmaf(col[a], r[b], acc[a]);
+            }
+#pragma unroll
+            for (int dh = 0; dh < K; ++dh)
+#pragma unroll
+                for (int dw = (dh == 0 ? 2 : 1); dw < K; ++dw)
+#pragma unroll
+                    for (int b = 0; b < C; ++b) {
+                        const int slot = (u - dw + 2 * KM) % KM;      // produced at step s - dw
+                        const float v = dh == 0 ? own[b][slot] : up[dh - 1][b][slot];
+                        float col[C];
+                        if constexpr (S::WREG) {
+#pragma unroll
+                            for (int a = 0; a < C; ++a) col[a] = Ar[((dh * K + dw) * C + b) * C + a];
+                        } else load_col<C>(As, (dh * K + dw) * C + b, col);
+                        if (((dh * K + dw) & 1) == 0) {
+#pragma unroll
+                            for (int a = 0; a < C; ++a) acc[a] = fmaf(-col[a], v, acc[a]);
+                        } else {
+#pragma unroll
+                            for (int a = 0; a < C; ++a) acc2[a] = fmaf(-col[a], v, acc2[a]);
+                        }
+                    }
+#pragma unroll
+            for (int a = 0; a < C; ++a) acc[a] += acc2[a];
+            // rows two and more above (their shuffles were fed by older results)
+#pragma unroll
+            for (int d = KM - 1; d >= 1; --d)
+#pragma unroll
+                for (int b = 0; b < C; ++b) {
+                    float col[C];
+                    if constexpr (S::WREG) {
+#pragma unroll
+                        for (int a = 0; a < C; ++a) col[a] = Ar[(((d + 1) * K) * C + b) * C + a];
+                    } else load_col<C>(As, ((d + 1) * K) * C + b, col);
+#pragma unroll
+                    for (int a = 0; a < C; ++a) acc[a] = fmaf(-col[a], nu[d][b], acc[a]);
+                }
+            // the two taps on the true critical path: left neighbour, then the row above
+#pragma unroll
+            for (int b = 0; b < C; ++b) {
+                float col[C];
+                if constexpr (S::WREG) {
+#pragma unroll
+                    for (int a = 0; a < C; ++a) col[a] = Ar[(1 * C + b) * C + a];
+                } else load_col<C>(As, 1 * C + b, col);
+#pragma unroll
+                for (int a = 0; a < C; ++a) acc[a] = fmaf(-col[a], own[b][(u - 1 + 2 * KM) % KM], acc[a]);
+            }
+#pragma unroll
+            for (int b = 0; b < C; ++b) {
+                float col[C];
+                if constexpr (S::WREG) {
+#pragma unroll
+                    for (int a = 0; a < C; ++a) col[a] = Ar[(K * C + b) * C + a];
+                } else load_col<C>(As, K * C + b, col);
+#pragma unroll
+                for (int a = 0; a < C; ++a) acc[a] = fmaf(-col[a], nu[0][b], acc[a]);
+            }
+            if (active) {
+#pragma unroll
+                for (int a = 0; a < C; ++a) img[a * HW + p] = acc[a];
+            }
+#pragma unroll
+            for (int b = 0; b < C; ++b) {
+                own[b][u] = active ? acc[b] : 0.f;
+#pragma unroll
+                for (int d = 0; d < KM; ++d) up[d][b][u] = nu[d][b];
+            }
+            p += sgn;
+        }
+        if constexpr (MULTI) {
+            if (((s0 + KM) & 7) == 0) {
+                __threadfence_block();
+                __syncwarp();
+                if (lane == 0) progress[j] = s0 + KM;
+            }
+        }
+    }
+    if constexpr (MULTI) {
+        __threadfence_block();
+        __syncwarp();
+        if (lane == 0) progress[j] = prod_steps;
+    }
+    return true;
+}
+
+// Sum v[0..31] over the 32 lanes; lane i returns the total of entry i.
+__device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane)
+{
+#pragma unroll
+    for (int off = 16, n = 32; off >= 1; off >>= 1, n >>= 1) {
+        const bool hi = (lane & off) != 0;
+#pragma unroll
+        for (int q = 0; q < n / 2; ++q) {
+            const float send = hi ? v[q] : v[q + n / 2];
+            const float keep = hi ? v[q + n / 2] : v[q];
+            v[q] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+    }
+    return v[0];
+}
+
+// grad_w partial of one row block, lane = column (Theorem 2 in closed form):
+//   part[((dh*K+dw)*C + co)*C + ci] = sum_{h in block, w} gy[co][h][w] * x[ci][h-dh][w-dw]
+// written to `dst` (shared memory, NA floats) by the lanes that end up owning each entry.
+template <int C, int K>
+__device__ __forceinline__ void grad_w_block(const float* gy, const float* xs, int H, int W, int j, int lane, float* dst)
+{
+    using S = WarpShape<C, K>;
+    constexpr int COB = S::COB;
+    constexpr int NACC = COB * C * K * K;
+    const int HW = H * W;
+    const int h0 = 32 * j, h1 = min(H, h0 + 32);
+    for (int co0 = 0; co0 < C; co0 += COB) {
+        float acc[NACC];
+#pragma unroll
+        for (int i = 0; i < NACC; ++i) acc[i] = 0.f;
+        for (int w0 = 0; w0 < W; w0 += 32) {
+            const int w = w0 + lane;
+            const bool col_ok = w < W;
+            float xr[K][C][K];       // [row slot][ci][dw] = x[ci][row][w-dw]
+#pragma unroll
+            for (int q = 1; q < K; ++q) {
+                const int row = h0 - q;
+#pragma unroll
+                for (int ci = 0; ci < C; ++ci)
+#pragma unroll
+                    for (int dw = 0; dw < K; ++dw)
+                        xr[(K - q) % K][ci][dw] = (row >= 0 && col_ok && w - dw >= 0) ? xs[ci * HW + row * W + w - dw] : 0.f;
+            }
+            for (int hb = h0; hb < h1; hb += K) {
+#pragma unroll
+                for (int r = 0; r < K; ++r) {
+                    const int h = hb + r;
+                    if (h < h1) {
+#pragma unroll
+                        for (int ci = 0; ci < C; ++ci)
+#pragma unroll
+                            for (int dw = 0; dw < K; ++dw)
+                                xr[r][ci][dw] = (col_ok && w - dw >= 0) ? xs[ci * HW + h * W + w - dw] : 0.f;
+                        float g[COB];
+#pragma unroll
+                        for (int c = 0; c < COB; ++c) g[c] = col_ok ? gy[(co0 + c) * HW + h * W + w] : 0.f;
+#pragma unroll
+                        for (int dh = 0; dh < K; ++dh)
+#pragma unroll
+                            for (int dw = 0; dw < K; ++dw)
+#pragma unroll
+                                for (int c = 0; c < COB; ++c)
+#pragma unroll
+                                    for (int ci = 0; ci < C; ++ci)
+                                        acc[((dh * K + dw) * COB + c) * C + ci] =
+                                            fmaf(g[c], xr[(r - dh + K) % K][ci][dw], acc[((dh * K + dw) * COB + c) * C + ci]);
+                    }
+                }
+            }
+        }
+        // cross-lane sums, 32 entries at a time
+#pragma unroll
+        for (int base = 0; base < NACC; base += 32) {
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = (base + i < NACC) ? acc[base + i] : 0.f;
+            const float tot = transpose_reduce32(v, lane);
+            const int i = base + lane;
+            if (i < NACC) {
+                const int ci = i % C, c = (i / C) % COB, tap = i / (C * COB);
+                dst[(tap * C + co0 + c) * C + ci] = tot;
+            }
+        }
+    }
+}
+
+// Float offsets of the kernel's shared-memory regions (all multiples of 32 floats = 128 bytes).
+template <int C, int K>
+struct WarpSmem {
+    using S = WarpShape<C, K>;
+    int as_off, bar_off, prog_off, red_off, img_off, imgf, total;
+    __host__ __device__ WarpSmem(int H, int W, int nb, int ipc, bool bwd)
+    {
+        auto up32 = [](int v) { return (v + 31) & ~31; };
+        as_off = 0;
+        bar_off = as_off + up32(S::NAP);
+        prog_off = bar_off + up32(2 * ipc);
+        red_off = prog_off + up32(ipc * nb);
+        img_off = red_off + (bwd ? up32(nb * ipc * S::NA) : 0);
+        imgf = up32(C * H * W);
+        total = img_off + imgf * ipc * (bwd ? 2 : 1);
+    }
+};
+
+template <int C, int K, bool BWD, bool MULTI>
+__global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
+{
+    using S = WarpShape<C, K>;
+    extern __shared__ __align__(128) float smem[];
+    const int H = p.H, W = p.W, HW = H * W, CHW = C * HW;
+    const int nwarps = blockDim.x >> 5;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int li = warp / p.nb, j = warp - li * p.nb;  // image within the CTA, row block within the image
+    const int n = blockIdx.x * p.ipc + li;             // image index
+    const bool has_img = n < p.B;
+    const WarpSmem<C, K> lay(H, W, p.nb, p.ipc, BWD);
+
+    float* As = smem + lay.as_off;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + lay.bar_off);
+    int* progress = reinterpret_cast<int*>(smem + lay.prog_off);               // [ipc][nb]
+    float* red = smem + lay.red_off;                                           // [nwarps][NA] (backward)
+    float* img = smem + lay.img_off + li * lay.imgf * (BWD ? 2 : 1);           // rhs -> solution, in place
+    float* xs = img + lay.imgf;                                                // backward: saved x
+
+    const bool want_gw = BWD && p.grad_w != nullptr;
+    const bool leader = has_img && j == 0 && lane == 0;
+    // the image's bulk copy goes out first; the kernel transform below overlaps its latency
+    if (leader && p.bulk) {
+        mbar_init(&bars[li], 1);
+        fence_mbar_init();
+        const unsigned bytes = (unsigned)CHW * 4u;
+        mbar_expect_tx(&bars[li], want_gw ? 2 * bytes : bytes);
+        bulk_g2s(img, p.rhs + (size_t)n * CHW, bytes, &bars[li]);
+        if (want_gw) bulk_g2s(xs, p.xsaved + (size_t)n * CHW, bytes, &bars[li]);
+    }
+    if (has_img && !p.bulk) {
+        const float* src = p.rhs + (size_t)n * CHW;
+        for (int i = j * 32 + lane; i < CHW; i += p.nb * 32) img[i] = __ldg(src + i);
+        if (want_gw) {
+            const float* xsrc = p.xsaved + (size_t)n * CHW;
+            for (int i = j * 32 + lane; i < CHW; i += p.nb * 32) xs[i] = __ldg(xsrc + i);
+        }
+    }
+    if (threadIdx.x < p.ipc * p.nb) progress[threadIdx.x] = 0;
+    build_transformed_kernel<C, K, BWD>(p.w, As);
+    __syncthreads();
+
+    bool ok = true;
+    if (has_img) {
+        if (p.bulk) ok = mbar_wait_bounded(&bars[li], 0);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok)
+            ok = wavefront_block<C, K, MULTI>(img, As, H, W, BWD ? HW - 1 : 0, BWD ? -1 : 1, j,
+                                              progress + li * p.nb, lane);
+        if (!ok && lane == 0) raise_status(INVCONV_TIMEOUT);
+    }
+    __syncthreads();
+
+    if (has_img) {
+        float* dst = p.out + (size_t)n * CHW;
+        if (p.bulk) {
+            if (leader) {
+                fence_proxy_async();
+                bulk_s2g(dst, img, (unsigned)CHW * 4u);
+                bulk_commit();
+            }
+        } else {
+            for (int i = j * 32 + lane; i < CHW; i += p.nb * 32) dst[i] = img[i];
+        }
+    }
+
+    if constexpr (BWD) {
+        if (want_gw) {
+            float* mine = red + warp * S::NA;
+            if (has_img) grad_w_block<C, K>(img, xs, H, W, j, lane, mine);
+            else for (int i = lane; i < S::NA; i += 32) mine[i] = 0.f;
+            __syncthreads();
+            float* cta_part = p.partials + (size_t)blockIdx.x * S::NA;
+            for (int i = threadIdx.x; i < S::NA; i += blockDim.x) {
+                float s = 0.f;
+                for (int wq = 0; wq < nwarps; ++wq) s += red[wq * S::NA + i];
+                __stcg(cta_part + i, s);
+            }
+            __threadfence();
+            __syncthreads();
+            __shared__ unsigned ticket;
+            if (threadIdx.x == 0) ticket = atomicAdd(p.counter, 1u);
+            __syncthreads();
+            if (ticket == gridDim.x - 1) {
+                __threadfence();
+                for (int i = threadIdx.x; i < S::NA; i += blockDim.x) {
+                    float s = 0.f;
+                    for (unsigned b = 0; b < gridDim.x; ++b) s += __ldcg(p.partials + (size_t)b * S::NA + i);
+                    const int ci = i % C, co = (i / C) % C, tap = i / (C * C);
+                    const int dh = tap / K, dw = tap % K;
+                    const bool masked_out = (tap == 0 && ci > co);
+                    p.grad_w[((co * C + ci) * K + (K - 1 - dh)) * K + (K - 1 - dw)] = masked_out ? 0.f : -s;
+                }
+                if (threadIdx.x == 0) *p.counter = 0u;
+            }
+        }
+    }
+    if (p.bulk && leader) bulk_wait_read0();
+}
+
+// Dynamic shared memory the kernel needs for a launch shape.
+template <int C, int K>
+inline size_t warp_kernel_smem(int H, int W, int nb, int ipc, bool bwd)
+{
+    return sizeof(float) * (size_t)WarpSmem<C, K>(H, W, nb, ipc, bwd).total;
+}
+
+}  // namespace invconv
