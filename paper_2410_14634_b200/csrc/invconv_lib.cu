@@ -13,6 +13,7 @@
 #include "generic_kernels.cuh"
 #include "probe_kernels.cuh"
 #include "warp_kernels.cuh"
+#include "team_kernels.cuh"
 
 using namespace invconv;
 
@@ -132,10 +133,89 @@ size_t warp_workspace_bytes(int B, int C, int H, int W, int k)
     return INVCONV_WS_CONTROL_BYTES + sizeof(float) * (size_t)pl.grid * C * C * k * k;
 }
 
+// ---------------------------------------------------------------- team family
+int sm_count()
+{
+    static std::atomic<int> cached{0};
+    int v = cached.load();
+    if (v > 0) return v;
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        return 148;            // B200; only used for planning when no device is present
+    }
+    cached.store(n);
+    return n;
+}
+
+TeamPlan team_plan(int B, int C, int H, int W, int k)
+{
+    if (team_prep_smem(C) > kMaxDynSmem) return TeamPlan{};
+    return plan_team(B > 0 ? B : 1, C, H, W, k, kMaxDynSmem, sm_count());
+}
+
+size_t team_workspace_bytes(int B, int C, int H, int W, int k)
+{
+    if (!team_plan(B, C, H, W, k).ok) return 0;
+    return INVCONV_WS_CONTROL_BYTES + sizeof(float) * (size_t)k * k * C * C;
+}
+
+template <int TA, int NGN, int NGC>
+int launch_team_inst(const TeamPlan& pl, const TeamParams& prm, cudaStream_t st)
+{
+    auto kern = team_wavefront_kernel<TA, NGN, NGC>;
+    const int rc = set_smem_limit(kern, pl.smem);
+    if (rc) return rc;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(pl.ncl * pl.R);
+    cfg.blockDim = dim3(pl.threads);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = pl.R; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
+    if (e != cudaSuccess) {
+        std::fprintf(stderr, "invconv: team launch failed: %s\n", cudaGetErrorString(e));
+        cudaGetLastError();
+        return INVCONV_CUDA_ERROR;
+    }
+    return check_launch();
+}
+
+// Transposed or plain solve through the team family; the transformed kernel goes to the workspace.
+int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, void* ws, cudaStream_t st)
+{
+    const TeamPlan pl = team_plan(g.B, g.C, g.H, g.W, g.k);
+    if (!pl.ok) return INVCONV_UNSUPPORTED;
+    float* A = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES);
+    {
+        const size_t sm = team_prep_smem(g.C);
+        auto kern = bwd ? team_prep_kernel<true> : team_prep_kernel<false>;
+        const int rc = set_smem_limit(kern, sm);
+        if (rc) return rc;
+        kern<<<g.k * g.k, 256, sm, st>>>(w, A, g.C, g.k);
+        const int rl = check_launch();
+        if (rl) return rl;
+    }
+    TeamParams prm;
+    prm.rhs = rhs; prm.A = A; prm.out = out;
+    prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W; prm.K = g.k;
+    prm.R = pl.R; prm.CA = pl.CA; prm.LG = pl.LG; prm.NS = pl.NS; prm.NPG = pl.NPG; prm.CS = pl.CS;
+    prm.PMAXS = pl.PMAXS; prm.rot = bwd ? 1 : 0; prm.ncl = pl.ncl;
+#define X(TT, GN_, GC_) \
+    if (pl.TA == TT && pl.NGN == GN_ && pl.NGC == GC_) return launch_team_inst<TT, GN_, GC_>(pl, prm, st);
+    X(3, 3, 1) X(3, 6, 2) X(3, 9, 1) X(4, 3, 1) X(4, 6, 2) X(4, 9, 1)
+#undef X
+    return INVCONV_UNSUPPORTED;
+}
+
 // ---------------------------------------------------------------- dispatch
 int auto_path(int B, int C, int H, int W, int k)
 {
     if (plan_warp(B > 0 ? B : 1, C, H, W, k, true).ok) return INVCONV_PATH_WARP;
+    if (team_plan(B, C, H, W, k).ok) return INVCONV_PATH_TEAM;
     return INVCONV_PATH_GENERIC;
 }
 
@@ -148,6 +228,7 @@ int resolve_path(int B, int C, int H, int W, int k)
 size_t workspace_bytes_for(int path, int B, int C, int H, int W, int k)
 {
     if (path == INVCONV_PATH_WARP) return warp_workspace_bytes(B, C, H, W, k);
+    if (path == INVCONV_PATH_TEAM) return team_workspace_bytes(B, C, H, W, k);
     return 0;
 }
 
@@ -162,6 +243,8 @@ int launch_forward(int path, const float* y, const float* w, float* x, Geom g,
         return check_launch();
     case INVCONV_PATH_WARP:
         return launch_warp(false, y, w, x, nullptr, nullptr, g, ws, st);
+    case INVCONV_PATH_TEAM:
+        return launch_team(false, y, w, x, g, ws, st);
     default:
         return INVCONV_UNSUPPORTED;
     }
@@ -186,6 +269,17 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
     }
     case INVCONV_PATH_WARP:
         return launch_warp(true, gx, w, gy, x, gw, g, ws, st);
+    case INVCONV_PATH_TEAM: {
+        if (g.B > 0) {
+            const int rc = launch_team(true, gx, w, gy, g, ws, st);
+            if (rc) return rc;
+        }
+        if (gw) {
+            generic_grad_w_kernel<<<g.C * g.C * g.k * g.k, 128, 0, st>>>(gy, x, gw, g);
+            return check_launch();
+        }
+        return INVCONV_OK;
+    }
     default:
         return INVCONV_UNSUPPORTED;
     }

@@ -132,6 +132,22 @@ __device__ void build_transformed_kernel(const float* __restrict__ w, float* As)
     }
 }
 
+// Sum v[0..31] over the 32 lanes; lane i returns the total of entry i.
+__device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane)
+{
+#pragma unroll
+    for (int off = 16, n = 32; off >= 1; off >>= 1, n >>= 1) {
+        const bool hi = (lane & off) != 0;
+#pragma unroll
+        for (int q = 0; q < n / 2; ++q) {
+            const float send = hi ? v[q] : v[q + n / 2];
+            const float keep = hi ? v[q + n / 2] : v[q];
+            v[q] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+    }
+    return v[0];
+}
+
 // The wavefront over one block of up to 32 rows.  Logical pixel (lh, lw) of
 // channel c lives at img[c*HW + origin + sgn*(lh*W + lw)] (sgn = -1 walks the
 // rotated image of the transposed solve).  Returns false if a wait gave up.
@@ -142,9 +158,17 @@ __device__ void build_transformed_kernel(const float* __restrict__ w, float* As)
 // inside the block (lane <= d for the row d+1 above) get zeroed copies of the
 // taps that read those rows when the block is the image's first, so the
 // shuffle result feeds the FMA directly with no select on the dependent chain.
-template <int C, int K, bool MULTI>
+//
+// GW = true (transposed solve only) also accumulates this block's share of
+// grad_w (Theorem 2 in closed form) on the fly:  with q the lane's pixel,
+//   part[tap][co][ci] += grad_y[co][q + delta] * x[ci][q],
+// where grad_y[q + delta] is exactly the solved neighbour the step already
+// holds in registers; it costs one shared-memory load of x[q] and K*K*C*C FMAs
+// off the dependent chain.  The partial sums go to gw_dst[(tap*C + co)*C + ci].
+template <int C, int K, bool MULTI, bool GW>
 __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int H, int W, int origin, int sgn,
-                                                int j, volatile int* progress, int lane)
+                                                int j, volatile int* progress, int lane,
+                                                const float* xs = nullptr, float* gw_dst = nullptr)
 {
     using S = WarpShape<C, K>;
     constexpr int KM = K - 1;
@@ -178,6 +202,9 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
 #pragma unroll
             for (int d = 0; d < KM; ++d) up[d][b][q] = 0.f;
         }
+    float gacc[GW ? S::NA : 1];
+#pragma unroll
+    for (int i = 0; i < (GW ? S::NA : 1); ++i) gacc[i] = 0.f;
     int p = origin + sgn * ((32 * j + lane) * W - lane);    // offset of (lh, lw) at step 0
     float rnext[C];
 #pragma unroll
@@ -203,6 +230,11 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
             float r[C];
 #pragma unroll
             for (int c = 0; c < C; ++c) r[c] = rnext[c];
+            float xq[GW ? C : 1];
+            if constexpr (GW) {
+#pragma unroll
+                for (int c = 0; c < C; ++c) xq[c] = active ? xs[c * HW + p] : 0.f;
+            }
             {
                 const bool act1 = (ulw + 1u) < Wl;
 #pragma unroll
@@ -300,6 +332,22 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
 #pragma unroll
                 for (int a = 0; a < C; ++a) img[a * HW + p] = acc[a];
             }
+            if constexpr (GW) {
+#pragma unroll
+                for (int dh = 0; dh < K; ++dh)
+#pragma unroll
+                    for (int dw = 0; dw < K; ++dw)
+#pragma unroll
+                        for (int b = 0; b < C; ++b) {
+                            const int slot = (u - dw + 2 * KM) % KM;
+                            const float nbr = dh == 0 ? (dw == 0 ? acc[b] : own[b][slot])
+                                                      : (dw == 0 ? nu[dh - 1][b] : up[dh - 1][b][slot]);
+#pragma unroll
+                            for (int c = 0; c < C; ++c)
+                                gacc[((dh * K + dw) * C + b) * C + c] =
+                                    fmaf(nbr, xq[c], gacc[((dh * K + dw) * C + b) * C + c]);
+                        }
+            }
 #pragma unroll
             for (int b = 0; b < C; ++b) {
                 own[b][u] = active ? acc[b] : 0.f;
@@ -321,23 +369,24 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
         __syncwarp();
         if (lane == 0) progress[j] = prod_steps;
     }
-    return true;
-}
-
-// Sum v[0..31] over the 32 lanes; lane i returns the total of entry i.
-__device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane)
-{
+    if constexpr (GW) {
+        // rows above the image never existed for the first lanes of the first block: drop what they gathered
 #pragma unroll
-    for (int off = 16, n = 32; off >= 1; off >>= 1, n >>= 1) {
-        const bool hi = (lane & off) != 0;
+        for (int dh = 1; dh < K; ++dh)
+            if (first_block && lane < dh) {
 #pragma unroll
-        for (int q = 0; q < n / 2; ++q) {
-            const float send = hi ? v[q] : v[q + n / 2];
-            const float keep = hi ? v[q + n / 2] : v[q];
-            v[q] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+                for (int i = 0; i < K * C * C; ++i) gacc[dh * K * C * C + i] = 0.f;
+            }
+#pragma unroll
+        for (int base = 0; base < S::NA; base += 32) {
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = (base + i < S::NA) ? gacc[base + i] : 0.f;
+            const float tot = transpose_reduce32(v, lane);
+            if (base + lane < S::NA) gw_dst[base + lane] = tot;
         }
     }
-    return v[0];
+    return true;
 }
 
 // grad_w partial of one row block, lane = column (Theorem 2 in closed form):
@@ -446,9 +495,11 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + lay.bar_off);
     int* progress = reinterpret_cast<int*>(smem + lay.prog_off);               // [ipc][nb]
     float* red = smem + lay.red_off;                                           // [nwarps][NA] (backward)
-    float* img = smem + lay.img_off + li * lay.imgf * (BWD ? 2 : 1);           // rhs -> solution, in place
-    float* xs = img + lay.imgf;                                                // backward: saved x
+    float* img = smem + lay.img_off + li * lay.imgf;                           // rhs -> solution, in place
+    float* xs_all = smem + lay.img_off + p.ipc * lay.imgf;                     // backward: the saved x images
+    float* xs = xs_all + li * lay.imgf;
 
+    constexpr bool FUSE_GW = (C == 1);      // few enough partial sums to ride along in the wavefront's registers
     const bool want_gw = BWD && p.grad_w != nullptr;
     const bool leader = has_img && j == 0 && lane == 0;
     // the image's bulk copy goes out first; the kernel transform below overlaps its latency
@@ -476,9 +527,14 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     if (has_img) {
         if (p.bulk) ok = mbar_wait_bounded(&bars[li], 0);
         ok = __all_sync(0xffffffffu, ok);
-        if (ok)
-            ok = wavefront_block<C, K, MULTI>(img, As, H, W, BWD ? HW - 1 : 0, BWD ? -1 : 1, j,
-                                              progress + li * p.nb, lane);
+        if (ok) {
+            if (BWD && FUSE_GW && want_gw)
+                ok = wavefront_block<C, K, MULTI, BWD && FUSE_GW>(img, As, H, W, HW - 1, -1, j, progress + li * p.nb,
+                                                                  lane, xs, red + warp * S::NA);
+            else
+                ok = wavefront_block<C, K, MULTI, false>(img, As, H, W, BWD ? HW - 1 : 0, BWD ? -1 : 1, j,
+                                                         progress + li * p.nb, lane);
+        }
         if (!ok && lane == 0) raise_status(INVCONV_TIMEOUT);
     }
     __syncthreads();
@@ -499,8 +555,8 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     if constexpr (BWD) {
         if (want_gw) {
             float* mine = red + warp * S::NA;
-            if (has_img) grad_w_block<C, K>(img, xs, H, W, j, lane, mine);
-            else for (int i = lane; i < S::NA; i += 32) mine[i] = 0.f;
+            if (!has_img || !ok) { for (int i = lane; i < S::NA; i += 32) mine[i] = 0.f; }
+            else if (!FUSE_GW) grad_w_block<C, K>(img, xs, H, W, j, lane, mine);
             __syncthreads();
             float* cta_part = p.partials + (size_t)blockIdx.x * S::NA;
             for (int i = threadIdx.x; i < S::NA; i += blockDim.x) {
@@ -514,10 +570,27 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
             if (threadIdx.x == 0) ticket = atomicAdd(p.counter, 1u);
             __syncthreads();
             if (ticket == gridDim.x - 1) {
+                // last CTA: sum the CTA partials in CTA order.  They are staged through the (now idle) shared
+                // memory of the saved-x images so that all threads have loads in flight at once.
                 __threadfence();
+                const int G = (int)gridDim.x;
+                const int chunk = min(G, (p.ipc * lay.imgf) / S::NA);
+                for (int b0 = 0; chunk > 0 && b0 < G; b0 += chunk) {
+                    const int nbk = min(chunk, G - b0);
+                    for (int idx = threadIdx.x; idx < nbk * S::NA; idx += blockDim.x)
+                        xs_all[idx] = __ldcg(p.partials + (size_t)b0 * S::NA + idx);
+                    __syncthreads();
+                    for (int i = threadIdx.x; i < S::NA; i += blockDim.x) {
+                        float s = b0 == 0 ? 0.f : red[i];
+                        for (int b = 0; b < nbk; ++b) s += xs_all[b * S::NA + i];
+                        red[i] = s;
+                    }
+                    __syncthreads();
+                }
                 for (int i = threadIdx.x; i < S::NA; i += blockDim.x) {
                     float s = 0.f;
-                    for (unsigned b = 0; b < gridDim.x; ++b) s += __ldcg(p.partials + (size_t)b * S::NA + i);
+                    if (chunk > 0) s = red[i];
+                    else for (int b = 0; b < G; ++b) s += __ldcg(p.partials + (size_t)b * S::NA + i);
                     const int ci = i % C, co = (i / C) % C, tap = i / (C * C);
                     const int dh = tap / K, dw = tap % K;
                     const bool masked_out = (tap == 0 && ci > co);
