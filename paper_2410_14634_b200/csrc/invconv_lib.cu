@@ -14,6 +14,7 @@
 #include "probe_kernels.cuh"
 #include "warp_kernels.cuh"
 #include "team_kernels.cuh"
+#include "gradw_kernels.cuh"
 
 using namespace invconv;
 
@@ -154,16 +155,57 @@ TeamPlan team_plan(int B, int C, int H, int W, int k)
     return plan_team(B > 0 ? B : 1, C, H, W, k, kMaxDynSmem, sm_count());
 }
 
+GradWPlan gradw_plan(int B, int C, int H, int W, int k)
+{
+    return plan_gradw(B, C, H, W, k, kMaxDynSmem / 2, sm_count());      // two CTAs per SM
+}
+
 size_t team_workspace_bytes(int B, int C, int H, int W, int k)
 {
     if (!team_plan(B, C, H, W, k).ok) return 0;
-    return INVCONV_WS_CONTROL_BYTES + sizeof(float) * (size_t)k * k * C * C;
+    const size_t na = sizeof(float) * (size_t)k * k * C * C;
+    const GradWPlan gp = gradw_plan(B, C, H, W, k);
+    return INVCONV_WS_CONTROL_BYTES + na + (gp.ok ? na * gp.nbc : 0);
 }
 
-template <int TA, int NGN, int NGC>
+template <int TC, int K>
+int launch_gradw_inst(const GradWPlan& gp, const GradWParams& prm, cudaStream_t st)
+{
+    auto kern = gradw_tile_kernel<TC, K>;
+    const int rc = set_smem_limit(kern, gp.smem);
+    if (rc) return rc;
+    kern<<<gp.grid, 256, gp.smem, st>>>(prm);
+    return check_launch();
+}
+
+// grad_w through the tiled correlation kernel; partial sums live behind the transformed kernel in the workspace.
+int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, cudaStream_t st)
+{
+    const GradWPlan gp = gradw_plan(g.B, g.C, g.H, g.W, g.k);
+    const bool aligned = ((reinterpret_cast<uintptr_t>(gy) | reinterpret_cast<uintptr_t>(x)) & 15) == 0;
+    if (!gp.ok || !aligned || g.B == 0) {
+        generic_grad_w_kernel<<<g.C * g.C * g.k * g.k, 128, 0, st>>>(gy, x, gw, g);
+        return check_launch();
+    }
+    const size_t na = (size_t)g.k * g.k * g.C * g.C;
+    GradWParams prm;
+    prm.gy = gy; prm.x = x;
+    prm.partials = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES) + na;
+    prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W; prm.nbc = gp.nbc; prm.tiles = gp.tiles; prm.plane = gp.plane;
+    int rc = INVCONV_UNSUPPORTED;
+#define X(TT, KK_) if (gp.TC == TT && g.k == KK_) rc = launch_gradw_inst<TT, KK_>(gp, prm, st);
+    X(1, 1) X(1, 2) X(1, 3) X(1, 5) X(3, 1) X(3, 2) X(3, 3) X(3, 5)
+#undef X
+    if (rc) return rc;
+    const int blocks = (int)((na + 255) / 256 < 4096 ? (na + 255) / 256 : 4096);
+    gradw_reduce_kernel<<<blocks, 256, 0, st>>>(prm.partials, gw, gp.nbc, g.C, g.k);
+    return check_launch();
+}
+
+template <int TA, int NG>
 int launch_team_inst(const TeamPlan& pl, const TeamParams& prm, cudaStream_t st)
 {
-    auto kern = team_wavefront_kernel<TA, NGN, NGC>;
+    auto kern = team_wavefront_kernel<TA, NG>;
     const int rc = set_smem_limit(kern, pl.smem);
     if (rc) return rc;
     cudaLaunchConfig_t cfg = {};
@@ -195,7 +237,7 @@ int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, 
         auto kern = bwd ? team_prep_kernel<true> : team_prep_kernel<false>;
         const int rc = set_smem_limit(kern, sm);
         if (rc) return rc;
-        kern<<<g.k * g.k, 256, sm, st>>>(w, A, g.C, g.k);
+        kern<<<g.k * g.k, 512, sm, st>>>(w, A, g.C, g.k);
         const int rl = check_launch();
         if (rl) return rl;
     }
@@ -204,9 +246,8 @@ int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, 
     prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W; prm.K = g.k;
     prm.R = pl.R; prm.CA = pl.CA; prm.LG = pl.LG; prm.NS = pl.NS; prm.NPG = pl.NPG; prm.CS = pl.CS;
     prm.PMAXS = pl.PMAXS; prm.rot = bwd ? 1 : 0; prm.ncl = pl.ncl;
-#define X(TT, GN_, GC_) \
-    if (pl.TA == TT && pl.NGN == GN_ && pl.NGC == GC_) return launch_team_inst<TT, GN_, GC_>(pl, prm, st);
-    X(3, 3, 1) X(3, 6, 2) X(3, 9, 1) X(4, 3, 1) X(4, 6, 2) X(4, 9, 1)
+#define X(TT, NG_) if (pl.TA == TT && pl.NG == NG_) return launch_team_inst<TT, NG_>(pl, prm, st);
+    X(6, 2) X(6, 4) X(6, 7) X(3, 2) X(3, 4) X(3, 7) X(3, 10) X(4, 2) X(4, 4) X(4, 7) X(4, 10)
 #undef X
     return INVCONV_UNSUPPORTED;
 }
@@ -274,10 +315,7 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
             const int rc = launch_team(true, gx, w, gy, g, ws, st);
             if (rc) return rc;
         }
-        if (gw) {
-            generic_grad_w_kernel<<<g.C * g.C * g.k * g.k, 128, 0, st>>>(gy, x, gw, g);
-            return check_launch();
-        }
+        if (gw) return launch_gradw(gy, x, gw, g, ws, st);
         return INVCONV_OK;
     }
     default:

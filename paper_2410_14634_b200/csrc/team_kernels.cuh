@@ -38,85 +38,113 @@ namespace cg = cooperative_groups;
 // recursion: 12x12 diagonal blocks by column-parallel substitution, then pairs
 // of blocks are merged,  [[X11, 0], [-X22 L21 X11, X22]],  doubling the block
 // size each level, so the depth is logarithmic in C.
-// Shared memory: 3*C*C floats.
+// Shared memory: three C x C matrices (rows padded to 16 bytes).
 // ---------------------------------------------------------------------------
 template <bool BWD>
-__global__ void __launch_bounds__(256) team_prep_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K)
+__global__ void __launch_bounds__(512) team_prep_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K)
 {
-    extern __shared__ float sm[];
-    float* Lm = sm;               // [C][C] masked centre tap
-    float* Li = sm + C * C;       // [C][C] its inverse
-    float* T = sm + 2 * C * C;    // scratch of the inversion, then the tap's kernel slice
+    extern __shared__ __align__(16) float sm[];
+    const int CP = (C + 3) & ~3;  // row pitch (16-byte rows)
+    float* Lm = sm;               // [C][CP] masked centre tap; later the tap's kernel slice T
+    float* Li = sm + C * CP;      // [C][CP] inverse, row-major
+    float* Sc = sm + 2 * C * CP;  // [C][CP] scratch of the merge steps; later the inverse transposed
     const int KK = K * K, ctr = KK - 1;
     const int tid = threadIdx.x, NT = blockDim.x;
     const int tap = blockIdx.x;
     const int dh = tap / K, dw = tap % K;
     const int t = (K - 1 - dh) * K + (K - 1 - dw);
 
-    for (int e = tid; e < C * C; e += NT) {
-        const int i = e / C, j = e % C;
-        Lm[e] = (j <= i) ? __ldg(w + (size_t)e * KK + ctr) : 0.f;
-        Li[e] = 0.f;
-    }
+    for (int i = tid / 32; i < C; i += NT / 32)
+        for (int j = tid % 32; j < CP; j += 32) {
+            Lm[i * CP + j] = (j <= i && j < C) ? __ldg(w + (size_t)(i * C + j) * KK + ctr) : 0.f;
+            Li[i * CP + j] = 0.f;
+        }
     __syncthreads();
     constexpr int NB0 = 12;
-    // diagonal blocks: thread -> (block, column)
-    for (int col = tid; col < C; col += NT) {
+    for (int col = tid; col < C; col += NT) {       // diagonal blocks, one thread per column
         const int o = col / NB0 * NB0, e1 = min(C, o + NB0);
-        Li[col * C + col] = 1.0f / Lm[col * C + col];
+        Li[col * CP + col] = 1.0f / Lm[col * CP + col];
         for (int i = col + 1; i < e1; ++i) {
             float s = 0.f;
-            for (int m = col; m < i; ++m) s += Lm[i * C + m] * Li[m * C + col];
-            Li[i * C + col] = -s / Lm[i * C + i];
+            for (int m = col; m < i; ++m) s = fmaf(Lm[i * CP + m], Li[m * CP + col], s);
+            Li[i * CP + col] = -s / Lm[i * CP + i];
         }
     }
     __syncthreads();
     for (int sz = NB0; sz < C; sz *= 2) {
-        // pairs (o, o+sz): rows [o+sz, min(o+2sz, C)), cols [o, o+sz)
-        // step 1: Tm = L21 * X11        (Tm stored at the X21 position of a scratch C x C matrix)
-        float* Tm = T;
-        for (int e = tid; e < C * C; e += NT) {
-            const int i = e / C, j = e % C;
-            const int o = i / (2 * sz) * (2 * sz);
-            if (i >= o + sz && j >= o && j < o + sz) {
+        // every pair of neighbouring blocks (o, o+sz): X21 = -X22 * (L21 * X11)
+        const int npairs = (C + 2 * sz - 1) / (2 * sz);
+        const int per = sz * sz;
+        for (int idx = tid; idx < npairs * per; idx += NT) {
+            const int pr = idx / per, rem = idx - pr * per;
+            const int ii = rem / sz, jj = rem - ii * sz;
+            const int o = pr * 2 * sz, i = o + sz + ii, j = o + jj;
+            if (i < C) {
                 float s = 0.f;
-                for (int m = j; m < o + sz; ++m) s += Lm[i * C + m] * Li[m * C + j];
-                Tm[e] = s;
+                for (int m = j; m < o + sz; ++m) s = fmaf(Lm[i * CP + m], Li[m * CP + j], s);
+                Sc[i * CP + j] = s;
             }
         }
         __syncthreads();
-        // step 2: X21 = -X22 * Tm
-        for (int e = tid; e < C * C; e += NT) {
-            const int i = e / C, j = e % C;
-            const int o = i / (2 * sz) * (2 * sz);
-            if (i >= o + sz && j >= o && j < o + sz) {
+        for (int idx = tid; idx < npairs * per; idx += NT) {
+            const int pr = idx / per, rem = idx - pr * per;
+            const int ii = rem / sz, jj = rem - ii * sz;
+            const int o = pr * 2 * sz, i = o + sz + ii, j = o + jj;
+            if (i < C) {
                 float s = 0.f;
-                for (int m = o + sz; m <= i; ++m) s += Li[i * C + m] * Tm[m * C + j];
-                Li[e] = -s;
+                for (int m = o + sz; m <= i; ++m) s = fmaf(Li[i * CP + m], Sc[m * CP + j], s);
+                Li[i * CP + j] = -s;
             }
         }
-        __syncthreads();
-    }
-    if (tap != 0) {
-        for (int e = tid; e < C * C; e += NT) T[e] = __ldg(w + (size_t)e * KK + t);     // T[m][b] = w[m][b][tap]
         __syncthreads();
     }
     float* out = A + (size_t)tap * C * C;
-    for (int e = tid; e < C * C; e += NT) {
-        const int b = e / C, a = e % C;
-        float v = 0.f;
-        if (tap == 0) {
-            v = BWD ? Li[b * C + a] : Li[a * C + b];
-        } else if (!BWD) {
-            for (int m = 0; m <= a; ++m) v += Li[a * C + m] * T[m * C + b];
-        } else {
-            for (int m = a; m < C; ++m) v += Li[m * C + a] * T[b * C + m];
+    if (tap == 0) {
+        for (int e = tid; e < C * C; e += NT) {
+            const int b = e / C, a = e - b * C;
+            out[e] = BWD ? Li[b * CP + a] : Li[a * CP + b];
         }
-        out[e] = v;
+        return;
+    }
+    // T[m][b] = w[m][b][tap]  (over Lm, which is no longer needed); the forward product wants L^-1 transposed
+    for (int i = tid / 32; i < C; i += NT / 32)
+        for (int j = tid % 32; j < CP; j += 32) {
+            Lm[i * CP + j] = j < C ? __ldg(w + (size_t)(i * C + j) * KK + t) : 0.f;
+            if (!BWD && j < C) Sc[j * CP + i] = Li[i * CP + j];
+        }
+    __syncthreads();
+    const float* T = Lm;
+    const int nq = CP / 4;
+    // thread -> (output channel a, quad of input channels b): conflict-free column reads, broadcast quads
+    for (int task = tid; task < C * nq; task += NT) {
+        const int bq = task / C, a = task - bq * C;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (!BWD) {
+            // A[b][a] = sum_{m <= a} Li[a][m] * T[m][b]
+            for (int m = 0; m <= a; ++m) {
+                const float l = Sc[m * CP + a];
+                const float4 tv = *reinterpret_cast<const float4*>(T + m * CP + bq * 4);
+                acc.x = fmaf(l, tv.x, acc.x); acc.y = fmaf(l, tv.y, acc.y);
+                acc.z = fmaf(l, tv.z, acc.z); acc.w = fmaf(l, tv.w, acc.w);
+            }
+        } else {
+            // A[b][a] = sum_{m >= a} Li[m][a] * T[b][m]
+            for (int m = a; m < C; ++m) {
+                const float l = Li[m * CP + a];
+                acc.x = fmaf(l, T[(bq * 4 + 0) * CP + m], acc.x);
+                acc.y = fmaf(l, (bq * 4 + 1 < C) ? T[(bq * 4 + 1) * CP + m] : 0.f, acc.y);
+                acc.z = fmaf(l, (bq * 4 + 2 < C) ? T[(bq * 4 + 2) * CP + m] : 0.f, acc.z);
+                acc.w = fmaf(l, (bq * 4 + 3 < C) ? T[(bq * 4 + 3) * CP + m] : 0.f, acc.w);
+            }
+        }
+        const float v[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (bq * 4 + q < C) out[(size_t)(bq * 4 + q) * C + a] = v[q];
     }
 }
 
-inline size_t team_prep_smem(int C) { return sizeof(float) * 3 * (size_t)C * C; }
+inline size_t team_prep_smem(int C) { return sizeof(float) * 3 * (size_t)C * ((C + 3) & ~3); }
 
 // ---------------------------------------------------------------------------
 struct TeamParams {
@@ -130,12 +158,18 @@ struct TeamParams {
     int NS;             // slices per pixel group (multiple of 32/LG)
     int NPG;            // pixel groups per CTA
     int CS;             // channel stride of the shared-memory images (multiple of 4)
-    int PMAXS;          // pixels one pixel group handles on the longest diagonal
+    int PMAXS;          // pixel slots of one pixel group on the longest diagonal (multiple of 4)
     int rot;            // 1: walk the image rotated by 180 degrees (transposed solve)
     int ncl;            // clusters in the grid
 };
 
-template <int TA, int NGN, int NGC>
+// Thread (pixel group pg, slice s, lane l) owns NG groups of four input channels
+// of one tap each and TA output channels.  Per diagonal it walks its pixels four
+// at a time: one broadcast 16-byte load per pixel and group, 16*TA FMAs.  The
+// slices' partial sums meet in shared memory; after one block barrier every
+// (pixel, channel) of the diagonal is summed over the slices and stored into
+// the image of every CTA of the cluster.
+template <int TA, int NG>
 __global__ void __launch_bounds__(256) team_wavefront_kernel(TeamParams p)
 {
     cg::cluster_group cluster = cg::this_cluster();
@@ -146,160 +180,137 @@ __global__ void __launch_bounds__(256) team_wavefront_kernel(TeamParams p)
     float* U = smem;
     float* RH = smem + IMG;
     float* red = smem + 2 * IMG;
-    const int r = (int)cluster.block_rank();
+    const int r = R > 1 ? (int)cluster.block_rank() : 0;
     const int cl = blockIdx.x / R;
     const int tid = threadIdx.x, NT = blockDim.x;
-    const int LG = p.LG, per_pg = p.NS * LG, NWP = per_pg >> 5;
+    const int LG = p.LG, NS = p.NS, per_pg = NS * LG;
     const int pg = tid / per_pg, tq = tid - pg * per_pg;
     const int s = tq / LG, l = tq - s * LG;
-    const int wq = tq >> 5;
     const int CAp = LG * TA;
     const int CB4 = CS >> 2;
-    const int GN = (K > 1 ? K * K - 2 : 1) * CB4, GC = (K > 1 ? 2 : 0) * CB4;
+    const int GT = K * K * CB4;
 
     // this thread's share of the transformed kernel, signs folded in
-    float wn[NGN][4][TA], wc[NGC][4][TA];
-    int offn[NGN], offc[NGC];
-    auto fetch = [&](int tap, int b4, float (&dst)[4][TA], int& off) {
-        const int dh = tap / K, dw = tap - dh * K;
-        off = (tap == 0 ? IMG : 0) - (dh * WP + dw) * CS + b4 * 4;
+    float wt[NG][4][TA];
+    int off[NG];
+#pragma unroll
+    for (int i = 0; i < NG; ++i) {
+        const int g = s + i * NS;
+        off[i] = 0;
+        if (g < GT) {
+            const int tap = g / CB4, b4 = g - tap * CB4;
+            const int dh = tap / K, dw = tap - dh * K;
+            off[i] = (tap == 0 ? IMG : 0) - (dh * WP + dw) * CS + b4 * 4;
+        }
 #pragma unroll
         for (int bb = 0; bb < 4; ++bb)
 #pragma unroll
             for (int t = 0; t < TA; ++t) {
-                const int b = b4 * 4 + bb, al = l * TA + t;
                 float v = 0.f;
-                if (b < C && al < CA) v = __ldg(p.A + ((size_t)tap * C + b) * C + r * CA + al);
-                dst[bb][t] = tap == 0 ? v : -v;
+                if (g < GT) {
+                    const int tap = g / CB4, b = (g - tap * CB4) * 4 + bb, al = l * TA + t;
+                    if (b < C && al < CA) v = __ldg(p.A + ((size_t)tap * C + b) * C + r * CA + al);
+                    if (tap != 0) v = -v;
+                }
+                wt[i][bb][t] = v;
             }
-    };
-#pragma unroll
-    for (int i = 0; i < NGN; ++i) {
-        const int g = s + i * p.NS;
-        if (g < GN) {
-            const int tnc = g / CB4, b4 = g - tnc * CB4;
-            const int tap = tnc == 0 ? 0 : (tnc <= K - 2 ? tnc + 1 : tnc + 2);   // skips taps 1 and K
-            fetch(tap, b4, wn[i], offn[i]);
-        } else {
-            offn[i] = 0;
-#pragma unroll
-            for (int bb = 0; bb < 4; ++bb)
-#pragma unroll
-                for (int t = 0; t < TA; ++t) wn[i][bb][t] = 0.f;
-        }
-    }
-#pragma unroll
-    for (int i = 0; i < NGC; ++i) {
-        const int g = s + i * p.NS;
-        if (g < GC) {
-            const int tcr = g / CB4, b4 = g - tcr * CB4;
-            fetch(tcr == 0 ? 1 : K, b4, wc[i], offc[i]);
-        } else {
-            offc[i] = 0;
-#pragma unroll
-            for (int bb = 0; bb < 4; ++bb)
-#pragma unroll
-                for (int t = 0; t < TA; ++t) wc[i][bb][t] = 0.f;
-        }
     }
     float* Urem[8];
 #pragma unroll
-    for (int rr = 0; rr < 8; ++rr) Urem[rr] = rr < R ? cluster.map_shared_rank(U, rr) : U;
+    for (int rr = 0; rr < 8; ++rr) Urem[rr] = (R > 1 && rr < R) ? cluster.map_shared_rank(U, rr) : U;
 
     for (int i = tid; i < 2 * IMG; i += NT) smem[i] = 0.f;     // zero padding (and the channel padding) once
     __syncthreads();
+
+    // finalize items of this thread walk (pixel, channel) pairs in steps of NT without divisions
+    const int fin_i0 = tid / CA, fin_a0 = tid - fin_i0 * CA;
+    const int fin_di = NT / CA, fin_da = NT - fin_di * CA;
 
     const int ND = H + W - 1;
     for (int n = cl; n < p.B; n += p.ncl) {
         // right-hand side of this image, all channels, rotated for the transposed solve
         const float* src = p.rhs + (size_t)n * C * HW;
-        for (int idx = tid; idx < C * HW; idx += NT) {
-            const int c = idx / HW, pp = idx - c * HW;
-            int h = pp / W, w = pp - h * W;
-            if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
-            RH[((h + K - 1) * WP + (w + K - 1)) * CS + c] = __ldg(src + idx);
+        for (int c = tid / 32; c < C; c += NT / 32) {
+            for (int pp = tid % 32; pp < HW; pp += 32) {
+                int h = pp / W, w = pp - h * W;
+                if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
+                RH[((h + K - 1) * WP + (w + K - 1)) * CS + c] = __ldg(src + c * HW + pp);
+            }
         }
-        cluster.sync();
+        if (R > 1) cluster.sync(); else __syncthreads();
 
         for (int d = 0; d < ND; ++d) {
             const int hlo = max(0, d - (W - 1));
             const int npix = min(H - 1, d) - hlo + 1;
-            for (int q = 0; pg + p.NPG * q < npix; q += 2) {
-                const int i1 = pg + p.NPG * q, i2 = i1 + p.NPG;
-                const bool has2 = i2 < npix;
-                const int h1 = hlo + i1, h2 = has2 ? hlo + i2 : h1;
-                const float* u1 = U + ((h1 + K - 1) * WP + (d - h1) + K - 1) * CS;
-                const float* u2 = U + ((h2 + K - 1) * WP + (d - h2) + K - 1) * CS;
-                float acc1[TA], acc2[TA];
+            for (int q0 = 0; pg + p.NPG * q0 < npix; q0 += 4) {
+                const float* up[4];
 #pragma unroll
-                for (int t = 0; t < TA; ++t) { acc1[t] = 0.f; acc2[t] = 0.f; }
-#pragma unroll
-                for (int g = 0; g < NGN; ++g) {
-                    const float4 x1 = *reinterpret_cast<const float4*>(u1 + offn[g]);
-                    const float4 x2 = *reinterpret_cast<const float4*>(u2 + offn[g]);
-#pragma unroll
-                    for (int t = 0; t < TA; ++t) {
-                        acc1[t] = fmaf(wn[g][0][t], x1.x, acc1[t]); acc2[t] = fmaf(wn[g][0][t], x2.x, acc2[t]);
-                        acc1[t] = fmaf(wn[g][1][t], x1.y, acc1[t]); acc2[t] = fmaf(wn[g][1][t], x2.y, acc2[t]);
-                        acc1[t] = fmaf(wn[g][2][t], x1.z, acc1[t]); acc2[t] = fmaf(wn[g][2][t], x2.z, acc2[t]);
-                        acc1[t] = fmaf(wn[g][3][t], x1.w, acc1[t]); acc2[t] = fmaf(wn[g][3][t], x2.w, acc2[t]);
-                    }
+                for (int x = 0; x < 4; ++x) {
+                    int i = pg + p.NPG * (q0 + x);
+                    if (i >= npix) i = pg;                    // padding slot: recompute a valid pixel, result unused
+                    const int h = hlo + i;
+                    up[x] = U + ((h + K - 1) * WP + (d - h) + K - 1) * CS;
                 }
+                float acc[4][TA];
 #pragma unroll
-                for (int g = 0; g < NGC; ++g) {
-                    const float4 x1 = *reinterpret_cast<const float4*>(u1 + offc[g]);
-                    const float4 x2 = *reinterpret_cast<const float4*>(u2 + offc[g]);
+                for (int x = 0; x < 4; ++x)
 #pragma unroll
-                    for (int t = 0; t < TA; ++t) {
-                        acc1[t] = fmaf(wc[g][0][t], x1.x, acc1[t]); acc2[t] = fmaf(wc[g][0][t], x2.x, acc2[t]);
-                        acc1[t] = fmaf(wc[g][1][t], x1.y, acc1[t]); acc2[t] = fmaf(wc[g][1][t], x2.y, acc2[t]);
-                        acc1[t] = fmaf(wc[g][2][t], x1.z, acc1[t]); acc2[t] = fmaf(wc[g][2][t], x2.z, acc2[t]);
-                        acc1[t] = fmaf(wc[g][3][t], x1.w, acc1[t]); acc2[t] = fmaf(wc[g][3][t], x2.w, acc2[t]);
-                    }
+                    for (int t = 0; t < TA; ++t) acc[x][t] = 0.f;
+#pragma unroll
+                for (int g = 0; g < NG; ++g) {
+                    float4 u[4];
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) u[x] = *reinterpret_cast<const float4*>(up[x] + off[g]);
+#pragma unroll
+                    for (int x = 0; x < 4; ++x)
+#pragma unroll
+                        for (int t = 0; t < TA; ++t) {
+                            acc[x][t] = fmaf(wt[g][0][t], u[x].x, acc[x][t]);
+                            acc[x][t] = fmaf(wt[g][1][t], u[x].y, acc[x][t]);
+                            acc[x][t] = fmaf(wt[g][2][t], u[x].z, acc[x][t]);
+                            acc[x][t] = fmaf(wt[g][3][t], u[x].w, acc[x][t]);
+                        }
                 }
-                // sum over the slices that share this warp
-                for (int o = LG; o < 32; o <<= 1) {
+                float* dst = red + ((size_t)((pg * p.PMAXS + q0) * NS + s)) * CAp + l * TA;
 #pragma unroll
-                    for (int t = 0; t < TA; ++t) {
-                        acc1[t] += __shfl_xor_sync(0xffffffffu, acc1[t], o);
-                        acc2[t] += __shfl_xor_sync(0xffffffffu, acc2[t], o);
-                    }
-                }
-                if ((tq & 31) < LG) {
-                    float* d1 = red + ((pg * NWP + wq) * p.PMAXS + q) * CAp + l * TA;
+                for (int x = 0; x < 4; ++x)
 #pragma unroll
-                    for (int t = 0; t < TA; ++t) d1[t] = acc1[t];
-                    if (has2) {
-#pragma unroll
-                        for (int t = 0; t < TA; ++t) d1[CAp + t] = acc2[t];
-                    }
-                }
+                    for (int t = 0; t < TA; ++t) dst[x * NS * CAp + t] = acc[x][t];
             }
             __syncthreads();
-            // finish the diagonal: sum the warps' partial sums, publish to every CTA of the cluster
-            for (int idx = tid; idx < npix * CA; idx += NT) {
-                const int i = idx / CA, al = idx - i * CA;
+            // finish the diagonal: sum the slices' partial sums, publish to every CTA of the cluster
+            for (int i = fin_i0, al = fin_a0; i < npix; ) {
                 const int pgi = i % p.NPG, q = i / p.NPG;
-                const float* src2 = red + ((pgi * NWP) * p.PMAXS + q) * CAp + al;
-                float v = 0.f;
-                for (int ww = 0; ww < NWP; ++ww) v += src2[ww * p.PMAXS * CAp];
+                const float* src2 = red + ((size_t)((pgi * p.PMAXS + q) * NS)) * CAp + al;
+                float v0 = 0.f, v1 = 0.f;
+                int ss = 0;
+                for (; ss + 1 < NS; ss += 2) { v0 += src2[ss * CAp]; v1 += src2[(ss + 1) * CAp]; }
+                if (ss < NS) v0 += src2[ss * CAp];
+                const float v = v0 + v1;
                 const int h = hlo + i;
-                const int off = ((h + K - 1) * WP + (d - h) + K - 1) * CS + r * CA + al;
+                const int o = ((h + K - 1) * WP + (d - h) + K - 1) * CS + r * CA + al;
+                if (R > 1) {
 #pragma unroll
-                for (int rr = 0; rr < 8; ++rr)
-                    if (rr < R) Urem[rr][off] = v;
+                    for (int rr = 0; rr < 8; ++rr)
+                        if (rr < R) Urem[rr][o] = v;
+                } else {
+                    U[o] = v;
+                }
+                i += fin_di; al += fin_da;
+                if (al >= CA) { al -= CA; ++i; }
             }
-            cluster.sync();
+            if (R > 1) cluster.sync(); else __syncthreads();
         }
         // write back this CTA's channels
         float* dst = p.out + (size_t)n * C * HW + (size_t)r * CA * HW;
-        for (int idx = tid; idx < CA * HW; idx += NT) {
-            const int al = idx / HW, pp = idx - al * HW;
-            int h = pp / W, w = pp - h * W;
-            if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
-            dst[idx] = U[((h + K - 1) * WP + (w + K - 1)) * CS + r * CA + al];
+        for (int al = tid / 32; al < CA; al += NT / 32) {
+            for (int pp = tid % 32; pp < HW; pp += 32) {
+                int h = pp / W, w = pp - h * W;
+                if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
+                dst[al * HW + pp] = U[((h + K - 1) * WP + (w + K - 1)) * CS + r * CA + al];
+            }
         }
-        cluster.sync();
+        if (R > 1) cluster.sync(); else __syncthreads();
     }
 }
 
@@ -308,7 +319,7 @@ __global__ void __launch_bounds__(256) team_wavefront_kernel(TeamParams p)
 // ---------------------------------------------------------------------------
 struct TeamPlan {
     bool ok = false;
-    int R = 1, CA = 0, TA = 3, LG = 0, NS = 0, NPG = 1, CS = 0, PMAXS = 0, NGN = 0, NGC = 0;
+    int R = 1, CA = 0, TA = 3, LG = 0, NS = 0, NPG = 1, CS = 0, PMAXS = 0, NG = 0;
     int threads = 0, ncl = 0;
     size_t smem = 0;
 };
@@ -324,41 +335,48 @@ inline TeamPlan plan_team(int B, int C, int H, int W, int K, size_t max_smem, in
     if ((long long)C * C * K * K / R > 30000) return best;
     while (R < 8 && (long long)B * R * 2 <= sm_count && divisible(R * 2)) R *= 2;
     const int CA = C / R;
-    const int TA = (CA % 3 == 0) ? 3 : 4;
-    int LG = 1;
-    while (LG * TA < CA) LG *= 2;
-    if (LG > 32) return best;
-    const int SPW = 32 / LG;
     const int CS = (C + 3) & ~3;
-    const int CB4 = CS / 4;
-    const int GN = (K > 1 ? K * K - 2 : 1) * CB4, GC = (K > 1 ? 2 : 0) * CB4;
-    const int menu[3][2] = {{3, 1}, {6, 2}, {9, 1}};
-    for (int m = 0; m < 3; ++m) {
-        const int NGN = menu[m][0], NGC = menu[m][1];
-        int NS = (GN + NGN - 1) / NGN;
-        if (GC > 0) NS = NS > (GC + NGC - 1) / NGC ? NS : (GC + NGC - 1) / NGC;
-        NS = (NS + SPW - 1) / SPW * SPW;
-        if (NS * LG > 256) continue;
-        TeamPlan pl;
-        pl.R = R; pl.CA = CA; pl.TA = TA; pl.LG = LG; pl.NS = NS; pl.CS = CS; pl.NGN = NGN; pl.NGC = NGC;
-        const int maxdiag = H < W ? H : W;
-        int NPG = 256 / (NS * LG);
-        if (NPG > maxdiag) NPG = maxdiag;
-        if (NPG < 1) NPG = 1;
-        pl.NPG = NPG;
-        pl.threads = NPG * NS * LG;
-        pl.PMAXS = ((maxdiag + NPG - 1) / NPG + 1) & ~1;       // pixel pairs: keep the slot count even
-        const size_t img = (size_t)(H + K - 1) * (W + K - 1) * CS;
-        const size_t red = (size_t)NPG * (NS * LG / 32) * pl.PMAXS * LG * TA;
-        pl.smem = sizeof(float) * (2 * img + red);
-        if (pl.smem > max_smem) continue;
-        int ncl = sm_count / R;
-        if (ncl > B) ncl = B;
-        if (ncl < 1) ncl = 1;
-        pl.ncl = ncl;
-        pl.ok = true;
-        best = pl;
-        break;
+    const int GT = K * K * (CS / 4);
+    const int maxdiag = H < W ? H : W;
+    const size_t img = (size_t)(H + K - 1) * (W + K - 1) * CS;
+    // candidates (TA, NG), cheapest register footprint first within each TA; prefer wide TA (more FMAs per load)
+    const int ta_opts[3] = {6, 3, 4};
+    const int ng_opts[4] = {2, 4, 7, 10};
+    for (int ti = 0; ti < 3 && !best.ok; ++ti) {
+        const int TA = ta_opts[ti];
+        if (TA == 6 && CA % 6 != 0) continue;
+        if (TA == 3 && CA % 3 != 0) continue;
+        int LG = 1;
+        while (LG * TA < CA) LG *= 2;
+        if (LG > 32) continue;
+        const int SPW = 32 / LG;
+        for (int ni = 0; ni < 4; ++ni) {
+            const int NG = ng_opts[ni];
+            if (NG * 4 * TA > 170) continue;                 // weights + accumulators must fit the register file
+            int NS = (GT + NG - 1) / NG;
+            NS = (NS + SPW - 1) / SPW * SPW;
+            if (NS * LG > 256) continue;
+            TeamPlan pl;
+            pl.R = R; pl.CA = CA; pl.TA = TA; pl.LG = LG; pl.NS = NS; pl.CS = CS; pl.NG = NG;
+            int NPG = 256 / (NS * LG);
+            const int want = (maxdiag + 3) / 4;               // no more pixel groups than batches of four pixels
+            if (NPG > want) NPG = want;
+            if (NPG < 1) NPG = 1;
+            pl.NPG = NPG;
+            pl.threads = NPG * NS * LG;
+            pl.PMAXS = (((maxdiag + NPG - 1) / NPG) + 3) & ~3;
+            const size_t red = (size_t)NPG * pl.PMAXS * NS * LG * TA;
+            pl.smem = sizeof(float) * (2 * img + red);
+            if (pl.smem > max_smem) continue;
+            int ncl = sm_count / R;
+            if (B * 2 > ncl * 3) ncl = (2 * sm_count) / R;   // many images: two resident clusters per SM hide barrier latency
+            if (ncl > B) ncl = B;
+            if (ncl < 1) ncl = 1;
+            pl.ncl = ncl;
+            pl.ok = true;
+            best = pl;
+            break;
+        }
     }
     return best;
 }
