@@ -34,6 +34,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("INVCONV_NVCC_FLAGS", "").split()      # e.g. -DINVCONV_TEAM_TIMING for development builds
     cmd += sources() + ["-o", tmp]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

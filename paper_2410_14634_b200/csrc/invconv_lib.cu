@@ -202,10 +202,10 @@ int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, c
     return check_launch();
 }
 
-template <int TA, int NG>
+template <int TA, int NGN, int NGC, int PM, int MAXT>
 int launch_team_inst(const TeamPlan& pl, const TeamParams& prm, cudaStream_t st)
 {
-    auto kern = team_wavefront_kernel<TA, NG>;
+    auto kern = team_wavefront_kernel<TA, NGN, NGC, PM, MAXT>;
     const int rc = set_smem_limit(kern, pl.smem);
     if (rc) return rc;
     cudaLaunchConfig_t cfg = {};
@@ -245,9 +245,16 @@ int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, 
     prm.rhs = rhs; prm.A = A; prm.out = out;
     prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W; prm.K = g.k;
     prm.R = pl.R; prm.CA = pl.CA; prm.LG = pl.LG; prm.NS = pl.NS; prm.NPG = pl.NPG; prm.CS = pl.CS;
-    prm.PMAXS = pl.PMAXS; prm.rot = bwd ? 1 : 0; prm.ncl = pl.ncl;
-#define X(TT, NG_) if (pl.TA == TT && pl.NG == NG_) return launch_team_inst<TT, NG_>(pl, prm, st);
-    X(6, 2) X(6, 4) X(6, 7) X(3, 2) X(3, 4) X(3, 7) X(3, 10) X(4, 2) X(4, 4) X(4, 7) X(4, 10)
+    prm.rot = bwd ? 1 : 0; prm.ncl = pl.ncl;
+    prm.vec = (((reinterpret_cast<uintptr_t>(rhs) | reinterpret_cast<uintptr_t>(out)) & 15) == 0 && (g.H * g.W) % 4 == 0) ? 1 : 0;
+    prm.div_w = make_fast_div((unsigned)g.W);
+    prm.div_hw = make_fast_div((unsigned)(g.H * g.W));
+    prm.div_q4 = make_fast_div((unsigned)(g.H * g.W / 4 > 0 ? g.H * g.W / 4 : 1));
+#define X(TT, GN_, GC_, PM_, MT_)                                                              \
+    if (pl.TA == TT && pl.NGN == GN_ && pl.NGC == GC_ && pl.PM == PM_ && pl.maxt == MT_)          \
+        return launch_team_inst<TT, GN_, GC_, PM_, MT_>(pl, prm, st);
+    X(3, 3, 1, 8, 256) X(3, 6, 2, 8, 256) X(3, 9, 1, 8, 256) X(3, 3, 1, 16, 256) X(3, 6, 2, 16, 256) X(3, 9, 1, 16, 256)
+    X(4, 3, 1, 8, 256) X(4, 6, 2, 8, 256) X(4, 9, 1, 8, 256) X(4, 3, 1, 16, 256) X(4, 6, 2, 16, 256) X(4, 9, 1, 16, 256)
 #undef X
     return INVCONV_UNSUPPORTED;
 }

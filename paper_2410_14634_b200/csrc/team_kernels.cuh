@@ -24,8 +24,11 @@
 #pragma once
 
 #include <cooperative_groups.h>
+#include <cstdio>
+#include <cstdlib>
 
 #include "common.cuh"
+#include "tma.cuh"
 
 namespace invconv {
 namespace cg = cooperative_groups;
@@ -43,7 +46,7 @@ namespace cg = cooperative_groups;
 template <bool BWD>
 __global__ void __launch_bounds__(512) team_prep_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K)
 {
-    extern __shared__ __align__(16) float sm[];
+    extern __shared__ __align__(128) float sm[];
     const int CP = (C + 3) & ~3;  // row pitch (16-byte rows)
     float* Lm = sm;               // [C][CP] masked centre tap; later the tap's kernel slice T
     float* Li = sm + C * CP;      // [C][CP] inverse, row-major
@@ -157,170 +160,330 @@ struct TeamParams {
     int LG;             // lanes per slice (power of two), LG*TA >= CA
     int NS;             // slices per pixel group (multiple of 32/LG)
     int NPG;            // pixel groups per CTA
-    int CS;             // channel stride of the shared-memory images (multiple of 4)
-    int PMAXS;          // pixel slots of one pixel group on the longest diagonal (multiple of 4)
+    int CS;             // floats per pixel in the shared-memory images: C rounded up to 4, padded to 4 mod 8
+                        // so that pixel-major accesses spread over the banks
     int rot;            // 1: walk the image rotated by 180 degrees (transposed solve)
+    int vec;            // 1: images are 16-byte aligned and H*W is a multiple of 4
+    FastDiv div_w, div_hw, div_q4;   // divisions by W, H*W and H*W/4
     int ncl;            // clusters in the grid
 };
 
-// Thread (pixel group pg, slice s, lane l) owns NG groups of four input channels
-// of one tap each and TA output channels.  Per diagonal it walks its pixels four
-// at a time: one broadcast 16-byte load per pixel and group, 16*TA FMAs.  The
-// slices' partial sums meet in shared memory; after one block barrier every
-// (pixel, channel) of the diagonal is summed over the slices and stored into
-// the image of every CTA of the cluster.
-template <int TA, int NG>
-__global__ void __launch_bounds__(256) team_wavefront_kernel(TeamParams p)
+// Phase timing for development builds (-DINVCONV_TEAM_TIMING): thread 0 of CTA 0 prints SM-clock totals per phase.
+#ifdef INVCONV_TEAM_TIMING
+#define TEAM_TT(i) do { if (tid == 0) { const long long now_ = clock64(); tacc_[i] += now_ - tlast_; tlast_ = now_; } } while (0)
+#else
+#define TEAM_TT(i) do { } while (0)
+#endif
+
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+// Thread (pixel group pg, slice s, lane l) owns a few groups of four input
+// channels of one tap each and TA output channels, split into the groups whose
+// tap reads the previous diagonal (taps (0,1) and (1,0): the only ones on the
+// dependent chain) and all the others, which read diagonals solved at least two
+// steps ago.  Per diagonal it first runs the second kind for its pixels -- this
+// overlaps the arrival of the previous diagonal -- then waits for that diagonal,
+// runs the first kind, folds the slices that share its warp by shuffles and
+// leaves one partial sum per warp in shared memory.  After one block barrier
+// every (pixel, channel) of the diagonal is summed over the warps and published:
+// a plain store into this CTA's image and an asynchronous store (st.async) into
+// the image of every other CTA of the cluster.  Each CTA owns two mbarriers
+// (even / odd diagonals): all of its threads arrive after publishing and its
+// peers' asynchronous stores are counted in bytes, so one wait covers both.
+template <int TA, int NGN, int NGC, int PM, int MAXT>
+__global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
 {
-    cg::cluster_group cluster = cg::this_cluster();
-    extern __shared__ __align__(16) float smem[];
+    extern __shared__ __align__(128) float smem[];
+    __shared__ unsigned long long bars[2];
+#ifdef INVCONV_TEAM_TIMING
+    const long long tstart_ = clock64();
+#endif
     const int C = p.C, H = p.H, W = p.W, K = p.K, CS = p.CS, R = p.R, CA = p.CA;
     const int HP = H + K - 1, WP = W + K - 1, HW = H * W;
     const int IMG = HP * WP * CS;
     float* U = smem;
     float* RH = smem + IMG;
     float* red = smem + 2 * IMG;
-    const int r = R > 1 ? (int)cluster.block_rank() : 0;
     const int cl = blockIdx.x / R;
+    const int r = blockIdx.x - cl * R;              // rank in the cluster (1-D clusters of R consecutive CTAs)
     const int tid = threadIdx.x, NT = blockDim.x;
-    const int LG = p.LG, NS = p.NS, per_pg = NS * LG;
+    const int LG = p.LG, NS = p.NS, per_pg = NS * LG, NPG = p.NPG;
     const int pg = tid / per_pg, tq = tid - pg * per_pg;
     const int s = tq / LG, l = tq - s * LG;
+    const int wq = tq >> 5, NWP = per_pg >> 5;
     const int CAp = LG * TA;
-    const int CB4 = CS >> 2;
-    const int GT = K * K * CB4;
+    const int CB4 = (C + 3) >> 2;
+    const int GN = (K > 1 ? K * K - 2 : 1) * CB4, GC = (K > 1 ? 2 : 0) * CB4;
+    const int DS = (WP - 1) * CS;                   // from one pixel of a diagonal to the next (one row down, one column left)
 
     // this thread's share of the transformed kernel, signs folded in
-    float wt[NG][4][TA];
-    int off[NG];
-#pragma unroll
-    for (int i = 0; i < NG; ++i) {
-        const int g = s + i * NS;
-        off[i] = 0;
-        if (g < GT) {
-            const int tap = g / CB4, b4 = g - tap * CB4;
-            const int dh = tap / K, dw = tap - dh * K;
-            off[i] = (tap == 0 ? IMG : 0) - (dh * WP + dw) * CS + b4 * 4;
-        }
+    float wn[NGN][4][TA], wc[NGC][4][TA];
+    int offn[NGN], offc[NGC];
+    auto fetch = [&](bool live, int tap, int b4, float (&dst)[4][TA], int& off) {
+        const int dh = tap / K, dw = tap - dh * K;
+        off = live ? (tap == 0 ? IMG : 0) - (dh * WP + dw) * CS + b4 * 4 : 0;
 #pragma unroll
         for (int bb = 0; bb < 4; ++bb)
 #pragma unroll
             for (int t = 0; t < TA; ++t) {
+                const int b = b4 * 4 + bb, al = l * TA + t;
                 float v = 0.f;
-                if (g < GT) {
-                    const int tap = g / CB4, b = (g - tap * CB4) * 4 + bb, al = l * TA + t;
-                    if (b < C && al < CA) v = __ldg(p.A + ((size_t)tap * C + b) * C + r * CA + al);
-                    if (tap != 0) v = -v;
-                }
-                wt[i][bb][t] = v;
+                if (live && b < C && al < CA) v = __ldg(p.A + ((size_t)tap * C + b) * C + r * CA + al);
+                dst[bb][t] = tap == 0 ? v : -v;
             }
-    }
-    float* Urem[8];
+    };
 #pragma unroll
-    for (int rr = 0; rr < 8; ++rr) Urem[rr] = (R > 1 && rr < R) ? cluster.map_shared_rank(U, rr) : U;
+    for (int i = 0; i < NGN; ++i) {
+        const int g = s + i * NS;
+        const int tnc = g / CB4, b4 = g - tnc * CB4;
+        const int tap = tnc == 0 ? 0 : (tnc <= K - 2 ? tnc + 1 : tnc + 2);   // skips taps 1 and K
+        fetch(g < GN, g < GN ? tap : 0, b4, wn[i], offn[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < NGC; ++i) {
+        const int g = s + i * NS;
+        const int tcr = g / CB4, b4 = g - tcr * CB4;
+        fetch(g < GC, g < GC ? (tcr == 0 ? 1 : K) : 0, b4, wc[i], offc[i]);
+    }
+    // peers' images and mbarriers (shared::cluster addresses)
+    uint32_t peerU[8], peerBar[8];
+#pragma unroll
+    for (int rr = 0; rr < 8; ++rr) {
+        const uint32_t rk = (uint32_t)(rr < R ? rr : r);
+        peerU[rr] = R > 1 ? cluster_map_u32(smem_u32(U), rk) : 0u;
+        peerBar[rr] = R > 1 ? cluster_map_u32(smem_u32(&bars[0]), rk) : 0u;
+    }
 
+    if (tid == 0) { mbar_init(&bars[0], NT >> 5); mbar_init(&bars[1], NT >> 5); fence_mbar_init(); }   // one arrival per warp
     for (int i = tid; i < 2 * IMG; i += NT) smem[i] = 0.f;     // zero padding (and the channel padding) once
     __syncthreads();
+    if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); }   // every CTA's barriers exist before anyone sends
 
     // finalize items of this thread walk (pixel, channel) pairs in steps of NT without divisions
     const int fin_i0 = tid / CA, fin_a0 = tid - fin_i0 * CA;
     const int fin_di = NT / CA, fin_da = NT - fin_di * CA;
 
+#ifdef INVCONV_TEAM_TIMING
+    long long tacc_[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long tlast_ = clock64();
+    if (threadIdx.x == 0 && blockIdx.x == 0) printf("team setup: %lld cycles\n", tlast_ - tstart_);
+#endif
     const int ND = H + W - 1;
-    for (int n = cl; n < p.B; n += p.ncl) {
-        // right-hand side of this image, all channels, rotated for the transposed solve
+    const int nq4 = HW >> 2;
+    unsigned stepno = 0;                            // diagonals processed so far by this CTA, across images
+    bool alive = true;
+    for (int n = cl; n < p.B && alive; n += p.ncl) {
+        TEAM_TT(7);
+        // right-hand side of this image, all channels, rotated for the transposed solve; the loads go out in
+        // batches of eight requests per thread so that their latency is paid once per batch
         const float* src = p.rhs + (size_t)n * C * HW;
-        for (int c = tid / 32; c < C; c += NT / 32) {
-            for (int pp = tid % 32; pp < HW; pp += 32) {
-                int h = pp / W, w = pp - h * W;
-                if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
-                RH[((h + K - 1) * WP + (w + K - 1)) * CS + c] = __ldg(src + c * HW + pp);
+        if (p.vec) {
+            const float4* src4 = reinterpret_cast<const float4*>(src);
+            const int nvec = C * nq4;
+            for (int v0 = tid; v0 < nvec; v0 += NT * 8) {
+                float4 tv[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (v0 + k * NT < nvec) tv[k] = __ldg(src4 + v0 + k * NT);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (v0 + k * NT < nvec) {
+                        const int vi = v0 + k * NT;
+                        const int c = fast_div(vi, p.div_q4), pp = (vi - c * nq4) << 2;
+                        const float vals[4] = {tv[k].x, tv[k].y, tv[k].z, tv[k].w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            int h = fast_div(pp + i, p.div_w), w = (pp + i) - h * W;
+                            if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
+                            RH[((h + K - 1) * WP + (w + K - 1)) * CS + c] = vals[i];
+                        }
+                    }
+                }
+            }
+        } else {
+            for (int e0 = tid; e0 < C * HW; e0 += NT * 8) {
+                float tv[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (e0 + k * NT < C * HW) tv[k] = __ldg(src + e0 + k * NT);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (e0 + k * NT < C * HW) {
+                        const int e = e0 + k * NT;
+                        const int c = fast_div(e, p.div_hw), pp = e - c * HW;
+                        int h = fast_div(pp, p.div_w), w = pp - h * W;
+                        if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
+                        RH[((h + K - 1) * WP + (w + K - 1)) * CS + c] = tv[k];
+                    }
+                }
             }
         }
-        if (R > 1) cluster.sync(); else __syncthreads();
+        __syncthreads();
+        TEAM_TT(0);
 
-        for (int d = 0; d < ND; ++d) {
+        for (int d = 0; d < ND; ++d, ++stepno) {
             const int hlo = max(0, d - (W - 1));
             const int npix = min(H - 1, d) - hlo + 1;
-            for (int q0 = 0; pg + p.NPG * q0 < npix; q0 += 4) {
-                const float* up[4];
+            // pixel i of the diagonal is (hlo + i, d - hlo - i); this thread's pixels are i = pg, pg + NPG, ...
+            const float* ubase = U + ((hlo + K - 1) * WP + (d - hlo) + K - 1) * CS + pg * DS;
+            const int qstep = NPG * DS;
+            float acc[PM][TA];
 #pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    int i = pg + p.NPG * (q0 + x);
-                    if (i >= npix) i = pg;                    // padding slot: recompute a valid pixel, result unused
-                    const int h = hlo + i;
-                    up[x] = U + ((h + K - 1) * WP + (d - h) + K - 1) * CS;
-                }
-                float acc[4][TA];
+            for (int q = 0; q < PM; ++q)
 #pragma unroll
-                for (int x = 0; x < 4; ++x)
+                for (int t = 0; t < TA; ++t) acc[q][t] = 0.f;
+            // taps that read diagonals <= d-2 (and the right-hand side)
 #pragma unroll
-                    for (int t = 0; t < TA; ++t) acc[x][t] = 0.f;
+            for (int q = 0; q < PM; q += 2) {
+                const int i0 = pg + NPG * q;
+                if (i0 < npix) {
+                    const float* u0 = ubase + q * qstep;
+                    const float* u1 = (i0 + NPG < npix) ? u0 + qstep : u0;
 #pragma unroll
-                for (int g = 0; g < NG; ++g) {
-                    float4 u[4];
-#pragma unroll
-                    for (int x = 0; x < 4; ++x) u[x] = *reinterpret_cast<const float4*>(up[x] + off[g]);
-#pragma unroll
-                    for (int x = 0; x < 4; ++x)
+                    for (int g = 0; g < NGN; ++g) {
+                        const float4 x0 = *reinterpret_cast<const float4*>(u0 + offn[g]);
+                        const float4 x1 = *reinterpret_cast<const float4*>(u1 + offn[g]);
 #pragma unroll
                         for (int t = 0; t < TA; ++t) {
-                            acc[x][t] = fmaf(wt[g][0][t], u[x].x, acc[x][t]);
-                            acc[x][t] = fmaf(wt[g][1][t], u[x].y, acc[x][t]);
-                            acc[x][t] = fmaf(wt[g][2][t], u[x].z, acc[x][t]);
-                            acc[x][t] = fmaf(wt[g][3][t], u[x].w, acc[x][t]);
+                            acc[q][t] = fmaf(wn[g][0][t], x0.x, acc[q][t]); acc[q + 1][t] = fmaf(wn[g][0][t], x1.x, acc[q + 1][t]);
+                            acc[q][t] = fmaf(wn[g][1][t], x0.y, acc[q][t]); acc[q + 1][t] = fmaf(wn[g][1][t], x1.y, acc[q + 1][t]);
+                            acc[q][t] = fmaf(wn[g][2][t], x0.z, acc[q][t]); acc[q + 1][t] = fmaf(wn[g][2][t], x1.z, acc[q + 1][t]);
+                            acc[q][t] = fmaf(wn[g][3][t], x0.w, acc[q][t]); acc[q + 1][t] = fmaf(wn[g][3][t], x1.w, acc[q + 1][t]);
                         }
+                    }
                 }
-                float* dst = red + ((size_t)((pg * p.PMAXS + q0) * NS + s)) * CAp + l * TA;
-#pragma unroll
-                for (int x = 0; x < 4; ++x)
-#pragma unroll
-                    for (int t = 0; t < TA; ++t) dst[x * NS * CAp + t] = acc[x][t];
             }
+            TEAM_TT(1);
+            // the previous diagonal: published by this CTA's threads and by the peers
+            if (d > 0) {
+                const unsigned prev = stepno - 1u;
+                if (!mbar_wait_bounded(&bars[prev & 1u], (prev >> 1) & 1u)) alive = false;
+            }
+            TEAM_TT(2);
+            // the two taps that read diagonal d-1
+#pragma unroll
+            for (int q = 0; q < PM; q += 2) {
+                const int i0 = pg + NPG * q;
+                if (i0 < npix) {
+                    const float* u0 = ubase + q * qstep;
+                    const float* u1 = (i0 + NPG < npix) ? u0 + qstep : u0;
+#pragma unroll
+                    for (int g = 0; g < NGC; ++g) {
+                        const float4 x0 = *reinterpret_cast<const float4*>(u0 + offc[g]);
+                        const float4 x1 = *reinterpret_cast<const float4*>(u1 + offc[g]);
+#pragma unroll
+                        for (int t = 0; t < TA; ++t) {
+                            acc[q][t] = fmaf(wc[g][0][t], x0.x, acc[q][t]); acc[q + 1][t] = fmaf(wc[g][0][t], x1.x, acc[q + 1][t]);
+                            acc[q][t] = fmaf(wc[g][1][t], x0.y, acc[q][t]); acc[q + 1][t] = fmaf(wc[g][1][t], x1.y, acc[q + 1][t]);
+                            acc[q][t] = fmaf(wc[g][2][t], x0.z, acc[q][t]); acc[q + 1][t] = fmaf(wc[g][2][t], x1.z, acc[q + 1][t]);
+                            acc[q][t] = fmaf(wc[g][3][t], x0.w, acc[q][t]); acc[q + 1][t] = fmaf(wc[g][3][t], x1.w, acc[q + 1][t]);
+                        }
+                    }
+                    // fold the slices that share this warp, then one partial sum per warp and pixel
+                    for (int o = LG; o < 32; o <<= 1) {
+#pragma unroll
+                        for (int t = 0; t < TA; ++t) {
+                            acc[q][t] += __shfl_xor_sync(0xffffffffu, acc[q][t], o);
+                            acc[q + 1][t] += __shfl_xor_sync(0xffffffffu, acc[q + 1][t], o);
+                        }
+                    }
+                    if ((tq & 31) < LG) {
+                        float* dst = red + ((size_t)i0 * NWP + wq) * CAp + l * TA;
+#pragma unroll
+                        for (int t = 0; t < TA; ++t) dst[t] = acc[q][t];
+                        if (i0 + NPG < npix) {
+#pragma unroll
+                            for (int t = 0; t < TA; ++t) dst[NPG * NWP * CAp + t] = acc[q + 1][t];
+                        }
+                    }
+                }
+            }
+            TEAM_TT(3);
             __syncthreads();
-            // finish the diagonal: sum the slices' partial sums, publish to every CTA of the cluster
+            TEAM_TT(4);
+            // finish the diagonal: sum the warps' partial sums and publish to every CTA of the cluster
+            unsigned long long* mybar = &bars[stepno & 1u];
+            if (R > 1 && tid == 0) mbar_expect_tx_only(mybar, (unsigned)((R - 1) * npix * CA * 4));
+            const int obase = ((hlo + K - 1) * WP + (d - hlo) + K - 1) * CS + r * CA;
             for (int i = fin_i0, al = fin_a0; i < npix; ) {
-                const int pgi = i % p.NPG, q = i / p.NPG;
-                const float* src2 = red + ((size_t)((pgi * p.PMAXS + q) * NS)) * CAp + al;
-                float v0 = 0.f, v1 = 0.f;
-                int ss = 0;
-                for (; ss + 1 < NS; ss += 2) { v0 += src2[ss * CAp]; v1 += src2[(ss + 1) * CAp]; }
-                if (ss < NS) v0 += src2[ss * CAp];
-                const float v = v0 + v1;
-                const int h = hlo + i;
-                const int o = ((h + K - 1) * WP + (d - h) + K - 1) * CS + r * CA + al;
+                const float* src2 = red + (size_t)i * NWP * CAp + al;
+                float v = 0.f;
+                for (int ww = 0; ww < NWP; ++ww) v += src2[ww * CAp];
+                const int o = obase + i * DS + al;
+                U[o] = v;
                 if (R > 1) {
 #pragma unroll
                     for (int rr = 0; rr < 8; ++rr)
-                        if (rr < R) Urem[rr][o] = v;
-                } else {
-                    U[o] = v;
+                        if (rr < R && rr != r)
+                            st_async_f32(peerU[rr] + 4u * (unsigned)o, v, peerBar[rr] + 8u * (stepno & 1u));
                 }
                 i += fin_di; al += fin_da;
                 if (al >= CA) { al -= CA; ++i; }
             }
-            if (R > 1) cluster.sync(); else __syncthreads();
+            __syncwarp();
+            if ((tid & 31) == 0) mbar_arrive(mybar);      // the warp's stores are ordered before its one arrival
+            TEAM_TT(5);
         }
+        {   // the last diagonal
+            const unsigned prev = stepno - 1u;
+            if (!mbar_wait_bounded(&bars[prev & 1u], (prev >> 1) & 1u)) alive = false;
+        }
+        TEAM_TT(6);
         // write back this CTA's channels
         float* dst = p.out + (size_t)n * C * HW + (size_t)r * CA * HW;
-        for (int al = tid / 32; al < CA; al += NT / 32) {
-            for (int pp = tid % 32; pp < HW; pp += 32) {
-                int h = pp / W, w = pp - h * W;
+        if (p.vec) {
+            float4* dst4 = reinterpret_cast<float4*>(dst);
+            for (int vi = tid; vi < CA * nq4; vi += NT) {
+                const int al = fast_div(vi, p.div_q4), pp = (vi - al * nq4) << 2;
+                float vals[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    int h = fast_div(pp + i, p.div_w), w = (pp + i) - h * W;
+                    if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
+                    vals[i] = U[((h + K - 1) * WP + (w + K - 1)) * CS + r * CA + al];
+                }
+                dst4[vi] = make_float4(vals[0], vals[1], vals[2], vals[3]);
+            }
+        } else {
+            for (int e = tid; e < CA * HW; e += NT) {
+                const int al = fast_div(e, p.div_hw), pp = e - al * HW;
+                int h = fast_div(pp, p.div_w), w = pp - h * W;
                 if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
-                dst[al * HW + pp] = U[((h + K - 1) * WP + (w + K - 1)) * CS + r * CA + al];
+                dst[e] = U[((h + K - 1) * WP + (w + K - 1)) * CS + r * CA + al];
             }
         }
-        if (R > 1) cluster.sync(); else __syncthreads();
+        // nobody publishes the next image's first diagonal into an image that is still being written back
+        if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
     }
+    if (!alive && tid == 0) raise_status(INVCONV_TIMEOUT);
+    if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); }   // no CTA exits while peers may still store into it
+#ifdef INVCONV_TEAM_TIMING
+    TEAM_TT(7);
+    if (tid == 0 && blockIdx.x == 0)
+        printf("team timing (cycles): load %lld | noncrit %lld | wait %lld | crit+red %lld | bar %lld | finalize %lld | lastwait %lld | store %lld\n",
+               tacc_[0], tacc_[1], tacc_[2], tacc_[3], tacc_[4], tacc_[5], tacc_[6], tacc_[7]);
+#endif
 }
 
 // ---------------------------------------------------------------------------
 // Host-side launch plan.
 // ---------------------------------------------------------------------------
+inline FastDiv make_fast_div(unsigned d)
+{
+    FastDiv f;
+    f.d = d;
+    unsigned sh = 0;
+    while ((1ull << sh) < d) ++sh;
+    f.shift = sh;
+    f.mul = (unsigned)((((1ull << sh) - d) << 32) / d + 1);
+    return f;
+}
+
 struct TeamPlan {
     bool ok = false;
-    int R = 1, CA = 0, TA = 3, LG = 0, NS = 0, NPG = 1, CS = 0, PMAXS = 0, NG = 0;
-    int threads = 0, ncl = 0;
+    int R = 1, CA = 0, TA = 3, LG = 0, NS = 0, NPG = 1, CS = 0, PM = 0, NGN = 0, NGC = 0;
+    int threads = 0, ncl = 0, maxt = 256;
     size_t smem = 0;
 };
 
@@ -334,49 +497,52 @@ inline TeamPlan plan_team(int B, int C, int H, int W, int K, size_t max_smem, in
     while (R < 8 && (long long)C * C * K * K / R > 30000 && divisible(R * 2)) R *= 2;
     if ((long long)C * C * K * K / R > 30000) return best;
     while (R < 8 && (long long)B * R * 2 <= sm_count && divisible(R * 2)) R *= 2;
+    if (const char* e = getenv("INVCONV_TEAM_R")) {           // measurement knob: force the cluster size
+        const int rr = atoi(e);
+        if (rr >= 1 && rr <= 8 && C % rr == 0) R = rr;
+    }
     const int CA = C / R;
-    const int CS = (C + 3) & ~3;
-    const int GT = K * K * (CS / 4);
+    const int CB4 = (C + 3) / 4;
+    int CS = CB4 * 4;
+    if (CS % 8 == 0) CS += 4;
+    const int GN = (K > 1 ? K * K - 2 : 1) * CB4, GC = (K > 1 ? 2 : 0) * CB4;
     const int maxdiag = H < W ? H : W;
     const size_t img = (size_t)(H + K - 1) * (W + K - 1) * CS;
-    // candidates (TA, NG), cheapest register footprint first within each TA; prefer wide TA (more FMAs per load)
-    const int ta_opts[3] = {6, 3, 4};
-    const int ng_opts[4] = {2, 4, 7, 10};
-    for (int ti = 0; ti < 3 && !best.ok; ++ti) {
-        const int TA = ta_opts[ti];
-        if (TA == 6 && CA % 6 != 0) continue;
-        if (TA == 3 && CA % 3 != 0) continue;
-        int LG = 1;
-        while (LG * TA < CA) LG *= 2;
-        if (LG > 32) continue;
-        const int SPW = 32 / LG;
-        for (int ni = 0; ni < 4; ++ni) {
-            const int NG = ng_opts[ni];
-            if (NG * 4 * TA > 170) continue;                 // weights + accumulators must fit the register file
-            int NS = (GT + NG - 1) / NG;
-            NS = (NS + SPW - 1) / SPW * SPW;
-            if (NS * LG > 256) continue;
-            TeamPlan pl;
-            pl.R = R; pl.CA = CA; pl.TA = TA; pl.LG = LG; pl.NS = NS; pl.CS = CS; pl.NG = NG;
-            int NPG = 256 / (NS * LG);
-            const int want = (maxdiag + 3) / 4;               // no more pixel groups than batches of four pixels
-            if (NPG > want) NPG = want;
-            if (NPG < 1) NPG = 1;
-            pl.NPG = NPG;
-            pl.threads = NPG * NS * LG;
-            pl.PMAXS = (((maxdiag + NPG - 1) / NPG) + 3) & ~3;
-            const size_t red = (size_t)NPG * pl.PMAXS * NS * LG * TA;
-            pl.smem = sizeof(float) * (2 * img + red);
-            if (pl.smem > max_smem) continue;
-            int ncl = sm_count / R;
-            if (B * 2 > ncl * 3) ncl = (2 * sm_count) / R;   // many images: two resident clusters per SM hide barrier latency
-            if (ncl > B) ncl = B;
-            if (ncl < 1) ncl = 1;
-            pl.ncl = ncl;
-            pl.ok = true;
-            best = pl;
-            break;
-        }
+    const int TA = (CA % 3 == 0) ? 3 : 4;
+    int LG = 1;
+    while (LG * TA < CA) LG *= 2;
+    if (LG > 32) return best;
+    const int SPW = 32 / LG;
+    const int menu[3][2] = {{3, 1}, {6, 2}, {9, 1}};
+    for (int m = 0; m < 3; ++m) {
+        const int NGN = menu[m][0], NGC = menu[m][1];
+        int NS = (GN + NGN - 1) / NGN;
+        if (GC > 0 && (GC + NGC - 1) / NGC > NS) NS = (GC + NGC - 1) / NGC;
+        NS = (NS + SPW - 1) / SPW * SPW;
+        const int maxt = 256;
+        if (NS * LG > maxt) continue;
+        TeamPlan pl;
+        pl.R = R; pl.CA = CA; pl.TA = TA; pl.LG = LG; pl.NS = NS; pl.CS = CS; pl.NGN = NGN; pl.NGC = NGC;
+        pl.maxt = maxt;
+        int NPG = maxt / (NS * LG);
+        const int want = (maxdiag + 1) / 2;                    // pixels are processed in pairs
+        if (NPG > want) NPG = want;
+        if (NPG < 1) NPG = 1;
+        const int per = (maxdiag + NPG - 1) / NPG;             // pixel slots per group on the longest diagonal
+        if (per > 16 || (maxt == 512 && per > 8)) continue;
+        pl.PM = per <= 8 ? 8 : 16;
+        pl.NPG = NPG;
+        pl.threads = NPG * NS * LG;
+        const size_t red = (size_t)(maxdiag + NPG) * (NS * LG / 32) * LG * TA;
+        pl.smem = sizeof(float) * (2 * img + red);
+        if (pl.smem > max_smem) continue;
+        int ncl = sm_count / R;
+        if (ncl > B) ncl = B;
+        if (ncl < 1) ncl = 1;
+        pl.ncl = ncl;
+        pl.ok = true;
+        best = pl;
+        break;
     }
     return best;
 }

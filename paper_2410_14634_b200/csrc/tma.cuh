@@ -71,4 +71,40 @@ __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.
 // Order generic-proxy writes to shared memory before later async-proxy (bulk copy) reads.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// Raise the pending byte count of the current phase without arriving.
+__device__ __forceinline__ void mbar_expect_tx_only(unsigned long long* bar, unsigned bytes)
+{
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// Address of this CTA's shared-memory location `local` in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_map_u32(uint32_t local, uint32_t rank)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    return remote;
+}
+
+// Asynchronous 4-byte store into a peer CTA's shared memory; the peer's mbarrier counts the bytes.
+__device__ __forceinline__ void st_async_f32(uint32_t remote_addr, float v, uint32_t remote_bar)
+{
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.u32 [%0], %1, [%2];" ::"r"(remote_addr),
+                 "r"(__float_as_uint(v)), "r"(remote_bar)
+                 : "memory");
+}
+
+// Division by a run-time constant through a precomputed multiplier (valid for n < 2^31).
+struct FastDiv {
+    unsigned mul, shift, d;
+};
+__device__ __forceinline__ int fast_div(int n, FastDiv f)
+{
+    return (int)((__umulhi((unsigned)n, f.mul) + (unsigned)n) >> f.shift);
+}
+
 }  // namespace invconv
