@@ -129,6 +129,38 @@ int invconv_step_host(const float* y_host, const float* w_host, const float* gra
                       int B, int C, int H, int W, int k,
                       void* device_scratch, size_t device_scratch_bytes, void* stream);
 
+/* invconv_backward for callers that must not allocate.  (The paper has no
+ * counterpart; this is a deployment convenience.)
+ *
+ * Some hosts freeze their device-memory map once start-up is over -- an
+ * inference server with a fixed memory plan, a real-time loop, a plug-in that
+ * runs inside another framework's callback -- and from then on may call
+ * neither cudaMalloc nor a pooled allocator.  The other backward entry points
+ * need scratch memory (a completion counter and per-CTA partial sums of
+ * grad_w) that either the library takes from the device's memory pool
+ * (invconv_backward) or the caller provides (invconv_backward_ws).  This
+ * variant keeps that scratch in a fixed array of INVCONV_NOALLOC_SCRATCH_BYTES
+ * that is part of the library image itself: every GPU that loads the library
+ * holds those bytes until the process exits, whether or not the call is used.
+ *
+ *  - Same arguments, outputs and arithmetic as invconv_backward; served by the
+ *    warp-shuffle kernel family only.  Shapes that family does not serve return
+ *    INVCONV_UNSUPPORTED; shapes whose scratch would exceed the fixed array
+ *    return INVCONV_WORKSPACE_TOO_SMALL.  Nothing is launched in either case.
+ *  - Calls cudaMalloc, cudaFree or any other allocating routine never.
+ *  - The first call on each device looks up the array's device address (with
+ *    that device current) and caches it; make that first call before any
+ *    stream capture begins on the device.
+ *  - All calls on a device share the one array.  Each call clears the control
+ *    words it relies on, on `stream`, before its kernel runs, so a call may
+ *    follow an aborted one; but two calls that overlap on the GPU (different
+ *    streams without ordering between them) race on the array and produce
+ *    garbage in grad_w.  Order them. */
+#define INVCONV_NOALLOC_SCRATCH_BYTES (1u << 20)
+int invconv_backward_noalloc(const float* grad_x, const float* x, const float* w,
+                             float* grad_y, float* grad_w,
+                             int B, int C, int H, int W, int k, void* stream);
+
 /* Force a kernel family for subsequent calls from this process (default AUTO).
  * Returns the previous setting. */
 int invconv_set_path(int path);

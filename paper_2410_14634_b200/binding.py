@@ -48,6 +48,8 @@ def lib() -> ctypes.CDLL:
         L.invconv_workspace_bytes.restype = sz
         L.invconv_forward_ws.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, vp, sz, vp]
         L.invconv_backward_ws.argtypes = [fp, fp, fp, fp, fp, ci, ci, ci, ci, ci, vp, sz, vp]
+        L.invconv_backward_noalloc.argtypes = [fp, fp, fp, fp, fp, ci, ci, ci, ci, ci, vp]
+        L.invconv_backward_noalloc.restype = ci
         L.invconv_step_scratch_bytes.argtypes = [ci] * 5
         L.invconv_step_scratch_bytes.restype = sz
         L.invconv_step_host.argtypes = [vp] * 7 + [ci] * 5 + [vp, sz, vp]
@@ -146,6 +148,26 @@ def invconv_backward(grad_x: torch.Tensor, x: torch.Tensor, w: torch.Tensor, nee
                                          ws.data_ptr() if ws is not None else None,
                                          ws.numel() if ws is not None else 0, sp), "invconv_backward")
     return gy, gw
+
+
+NOALLOC_SCRATCH_BYTES = 1 << 20
+
+
+def invconv_backward_noalloc(grad_x: torch.Tensor, x: torch.Tensor, w: torch.Tensor,
+                             out_grad_y: torch.Tensor, out_grad_w: torch.Tensor,
+                             stream: Optional[torch.cuda.Stream] = None) -> None:
+    """`invconv_backward` for hosts that may no longer allocate device memory (a server with a frozen
+    memory plan, a callback inside another framework): the caller passes every buffer, outputs included, and
+    the library's scratch is a fixed array inside the library image (`NOALLOC_SCRATCH_BYTES`, shared by all
+    calls on a device -- do not let two calls overlap on the GPU).  Raises `InvConvError` with status
+    UNSUPPORTED or WORKSPACE_TOO_SMALL for shapes it does not serve; see `include/invconv.h`."""
+    _act(grad_x, "grad_x"); _act(x, "x"); _act(out_grad_y, "out_grad_y")
+    B, C, H, W = x.shape
+    k = _kern(w, C)
+    with torch.cuda.device(x.device):
+        _check(lib().invconv_backward_noalloc(grad_x.data_ptr(), x.data_ptr(), w.data_ptr(), out_grad_y.data_ptr(),
+                                              out_grad_w.data_ptr(), B, C, H, W, k, _stream_ptr(stream, x.device)),
+               "invconv_backward_noalloc")
 
 
 def masked_conv_forward(x: torch.Tensor, w: torch.Tensor, out: Optional[torch.Tensor] = None,

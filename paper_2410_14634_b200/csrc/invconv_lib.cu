@@ -488,6 +488,53 @@ int invconv_step_host(const float* y_host, const float* w_host, const float* gra
     return INVCONV_OK;
 }
 
+// ---------------------------------------------------------------- no-allocation backward
+// Scratch of invconv_backward_noalloc: part of the module image, one copy per device that loads it.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[INVCONV_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::atomic<void*> g_noalloc_ptr[kMaxDevices];
+
+// Device address of the scratch array on the current device.  In host code the array's name is only a
+// handle for the runtime, not an address a kernel could use, so the address is asked for once per device.
+int noalloc_scratch(void** out)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return INVCONV_CUDA_ERROR; }
+    void* p = g_noalloc_ptr[dev].load();
+    if (!p) {
+        const cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess || !p) {
+            std::fprintf(stderr, "invconv: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
+            cudaGetLastError();
+            return INVCONV_CUDA_ERROR;
+        }
+        g_noalloc_ptr[dev].store(p);
+    }
+    *out = p;
+    return INVCONV_OK;
+}
+}  // namespace
+
+int invconv_backward_noalloc(const float* grad_x, const float* x, const float* w, float* grad_y, float* grad_w,
+                             int B, int C, int H, int W, int k, void* stream)
+{
+    const int rc = check_shape(B, C, H, W, k);
+    if (rc) return rc;
+    if (B == 0) return invconv_backward_ws(grad_x, x, w, grad_y, grad_w, B, C, H, W, k, nullptr, 0, stream);
+    if (!grad_x || !x || !w || !grad_y || grad_x == grad_y || x == grad_y) return INVCONV_BAD_ARG;
+    if (!plan_warp(B, C, H, W, k, true).ok) return INVCONV_UNSUPPORTED;
+    const size_t need = warp_workspace_bytes(B, C, H, W, k);
+    if (need > INVCONV_NOALLOC_SCRATCH_BYTES) return INVCONV_WORKSPACE_TOO_SMALL;
+    void* scratch = nullptr;
+    const int rs = noalloc_scratch(&scratch);
+    if (rs) return rs;
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemsetAsync(scratch, 0, INVCONV_WS_CONTROL_BYTES, st) != cudaSuccess) { cudaGetLastError(); return INVCONV_CUDA_ERROR; }
+    return launch_warp(true, grad_x, w, grad_y, x, grad_w, Geom{B, C, H, W, k}, scratch, st);
+}
+
 int invconv_set_path(int path)
 {
     if (path < INVCONV_PATH_AUTO || path > INVCONV_PATH_TEAM) return -1;
