@@ -178,7 +178,10 @@ int invconv_get_status(void* stream, int* device_status_out);
  * for a communication mechanism, with no other work on the chain:
  *   mechanism 0: warp shuffle + one FMA (lane = image row);
  *   mechanism 1: shared-memory store, block barrier, load, one FMA;
- *   mechanism 2: store to a cluster peer's shared memory, cluster barrier, load, one FMA.
+ *   mechanism 2: store to a cluster peer's shared memory, cluster barrier, load, one FMA;
+ *   mechanism 3: one dependent FMA (the latency of a single accumulator);
+ *   mechanism 4: two broadcast 16-byte shared-memory loads feeding 24 FMAs on six accumulators
+ *                (one "group" of the wide-channel kernels' inner loop, 8 warps resident).
  * Runs a chain of `steps` dependent steps in one CTA (cluster of 2 for 2) and
  * writes the elapsed SM clock cycles to cycles_out[0] and the chain's final
  * value to cycles_out[1] (device pointer to two 64-bit words).  Used for the

@@ -226,6 +226,30 @@ int launch_team_inst(const TeamPlan& pl, const TeamParams& prm, cudaStream_t st)
     return check_launch();
 }
 
+template <int TA, int NGN, int NGC, int PJ>
+int launch_pixel_inst(const TeamPlan& pl, const TeamParams& prm, cudaStream_t st)
+{
+    auto kern = team_pixel_kernel<TA, NGN, NGC, PJ>;
+    const int rc = set_smem_limit(kern, pl.smem);
+    if (rc) return rc;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(pl.ncl * pl.R);
+    cfg.blockDim = dim3(pl.threads);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = pl.R; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
+    if (e != cudaSuccess) {
+        std::fprintf(stderr, "invconv: pixel-team launch failed: %s\n", cudaGetErrorString(e));
+        cudaGetLastError();
+        return INVCONV_CUDA_ERROR;
+    }
+    return check_launch();
+}
+
 // Transposed or plain solve through the team family; the transformed kernel goes to the workspace.
 int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, void* ws, cudaStream_t st)
 {
@@ -245,11 +269,20 @@ int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, 
     prm.rhs = rhs; prm.A = A; prm.out = out;
     prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W; prm.K = g.k;
     prm.R = pl.R; prm.CA = pl.CA; prm.LG = pl.LG; prm.NS = pl.NS; prm.NPG = pl.NPG; prm.CS = pl.CS;
+    prm.KW = pl.KW;
     prm.rot = bwd ? 1 : 0; prm.ncl = pl.ncl;
     prm.vec = (((reinterpret_cast<uintptr_t>(rhs) | reinterpret_cast<uintptr_t>(out)) & 15) == 0 && (g.H * g.W) % 4 == 0) ? 1 : 0;
     prm.div_w = make_fast_div((unsigned)g.W);
     prm.div_hw = make_fast_div((unsigned)(g.H * g.W));
     prm.div_q4 = make_fast_div((unsigned)(g.H * g.W / 4 > 0 ? g.H * g.W / 4 : 1));
+    if (pl.pixel) {
+#define XP(TT, GN_, GC_, PJ_) \
+    if (pl.TA == TT && pl.NGN == GN_ && pl.NGC == GC_ && pl.PJ == PJ_) return launch_pixel_inst<TT, GN_, GC_, PJ_>(pl, prm, st);
+        XP(3, 3, 1, 1) XP(3, 6, 2, 1) XP(3, 12, 3, 1) XP(3, 3, 1, 2) XP(3, 6, 2, 2) XP(3, 12, 3, 2)
+        XP(4, 3, 1, 1) XP(4, 6, 2, 1) XP(4, 12, 3, 1) XP(4, 3, 1, 2) XP(4, 6, 2, 2) XP(4, 12, 3, 2)
+#undef XP
+        return INVCONV_UNSUPPORTED;
+    }
 #define X(TT, GN_, GC_, PM_, MT_)                                                              \
     if (pl.TA == TT && pl.NGN == GN_ && pl.NGC == GC_ && pl.PM == PM_ && pl.maxt == MT_)          \
         return launch_team_inst<TT, GN_, GC_, PM_, MT_>(pl, prm, st);
@@ -568,6 +601,8 @@ int invconv_probe_step_latency(int mechanism, int steps, unsigned long long* cyc
     switch (mechanism) {
     case 0: probe_shuffle_chain<<<1, 32, 0, st>>>(steps, cycles_out); break;
     case 1: probe_smem_chain<<<1, 256, 0, st>>>(steps, cycles_out); break;
+    case 3: probe_fma_chain<<<1, 32, 0, st>>>(steps, cycles_out); break;
+    case 4: probe_group_chain<<<1, 256, 0, st>>>(steps, cycles_out); break;
     case 2: {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2); cfg.blockDim = dim3(128); cfg.stream = st;

@@ -69,4 +69,47 @@ __global__ void __launch_bounds__(128) probe_cluster_chain(int steps, unsigned l
     }
 }
 
+// Mechanism 3: one dependent FMA chain (the latency of a single accumulator).
+__global__ void probe_fma_chain(int steps, unsigned long long* out)
+{
+    float a = 1.0f + 0.001f * threadIdx.x;
+    const float w = 0.999f, c = 0.001f;
+    const long long t0 = clock64();
+#pragma unroll 16
+    for (int i = 0; i < steps; ++i) a = fmaf(a, w, c);
+    const long long t1 = clock64();
+    if (threadIdx.x == 0) { out[0] = (unsigned long long)(t1 - t0); out[1] = (unsigned long long)__float_as_uint(a); }
+}
+
+// Mechanism 4: a broadcast 16-byte shared-memory load feeding twelve FMAs on six accumulators (one group of
+// the wide-channel kernels' inner loop); cycles per group.
+__global__ void probe_group_chain(int steps, unsigned long long* out)
+{
+    __shared__ __align__(16) float buf[1024];
+    for (int i = threadIdx.x; i < 1024; i += blockDim.x) buf[i] = 0.001f * i;
+    __syncthreads();
+    float acc[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    float w[12];
+#pragma unroll
+    for (int i = 0; i < 12; ++i) w[i] = 0.01f * (i + 1) + 0.0001f * threadIdx.x;
+    const int lane_off = (threadIdx.x >> 3) * 4;
+    const long long t0 = clock64();
+#pragma unroll 4
+    for (int i = 0; i < steps; ++i) {
+        const float4 x0 = *reinterpret_cast<const float4*>(buf + ((i * 8 + lane_off) & 1015));
+        const float4 x1 = *reinterpret_cast<const float4*>(buf + ((i * 8 + lane_off + 4) & 1015));
+        acc[0] = fmaf(w[0], x0.x, acc[0]); acc[1] = fmaf(w[1], x0.x, acc[1]); acc[2] = fmaf(w[2], x0.x, acc[2]);
+        acc[3] = fmaf(w[0], x1.x, acc[3]); acc[4] = fmaf(w[1], x1.x, acc[4]); acc[5] = fmaf(w[2], x1.x, acc[5]);
+        acc[0] = fmaf(w[3], x0.y, acc[0]); acc[1] = fmaf(w[4], x0.y, acc[1]); acc[2] = fmaf(w[5], x0.y, acc[2]);
+        acc[3] = fmaf(w[3], x1.y, acc[3]); acc[4] = fmaf(w[4], x1.y, acc[4]); acc[5] = fmaf(w[5], x1.y, acc[5]);
+        acc[0] = fmaf(w[6], x0.z, acc[0]); acc[1] = fmaf(w[7], x0.z, acc[1]); acc[2] = fmaf(w[8], x0.z, acc[2]);
+        acc[3] = fmaf(w[6], x1.z, acc[3]); acc[4] = fmaf(w[7], x1.z, acc[4]); acc[5] = fmaf(w[8], x1.z, acc[5]);
+        acc[0] = fmaf(w[9], x0.w, acc[0]); acc[1] = fmaf(w[10], x0.w, acc[1]); acc[2] = fmaf(w[11], x0.w, acc[2]);
+        acc[3] = fmaf(w[9], x1.w, acc[3]); acc[4] = fmaf(w[10], x1.w, acc[4]); acc[5] = fmaf(w[11], x1.w, acc[5]);
+    }
+    const long long t1 = clock64();
+    float s = acc[0] + acc[1] + acc[2] + acc[3] + acc[4] + acc[5];
+    if (threadIdx.x == 0) { out[0] = (unsigned long long)(t1 - t0); out[1] = (unsigned long long)__float_as_uint(s); }
+}
+
 }  // namespace invconv

@@ -159,7 +159,8 @@ struct TeamParams {
     int CA;             // output channels per CTA (C / R)
     int LG;             // lanes per slice (power of two), LG*TA >= CA
     int NS;             // slices per pixel group (multiple of 32/LG)
-    int NPG;            // pixel groups per CTA
+    int NPG;            // pixel groups per CTA (pixel-team variant: teams per CTA)
+    int KW;             // pixel-team variant: warps per team
     int CS;             // floats per pixel in the shared-memory images: C rounded up to 4, padded to 4 mod 8
                         // so that pixel-major accesses spread over the banks
     int rot;            // 1: walk the image rotated by 180 degrees (transposed solve)
@@ -340,18 +341,25 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
                 if (i0 < npix) {
                     const float* u0 = ubase + q * qstep;
                     const float* u1 = (i0 + NPG < npix) ? u0 + qstep : u0;
+                    // all loads first, then FMAs ordered so that neighbours in the instruction stream hit
+                    // different accumulators (2*TA independent chains)
+                    float xa[NGN][4], xb[NGN][4];
 #pragma unroll
                     for (int g = 0; g < NGN; ++g) {
                         const float4 x0 = *reinterpret_cast<const float4*>(u0 + offn[g]);
                         const float4 x1 = *reinterpret_cast<const float4*>(u1 + offn[g]);
-#pragma unroll
-                        for (int t = 0; t < TA; ++t) {
-                            acc[q][t] = fmaf(wn[g][0][t], x0.x, acc[q][t]); acc[q + 1][t] = fmaf(wn[g][0][t], x1.x, acc[q + 1][t]);
-                            acc[q][t] = fmaf(wn[g][1][t], x0.y, acc[q][t]); acc[q + 1][t] = fmaf(wn[g][1][t], x1.y, acc[q + 1][t]);
-                            acc[q][t] = fmaf(wn[g][2][t], x0.z, acc[q][t]); acc[q + 1][t] = fmaf(wn[g][2][t], x1.z, acc[q + 1][t]);
-                            acc[q][t] = fmaf(wn[g][3][t], x0.w, acc[q][t]); acc[q + 1][t] = fmaf(wn[g][3][t], x1.w, acc[q + 1][t]);
-                        }
+                        xa[g][0] = x0.x; xa[g][1] = x0.y; xa[g][2] = x0.z; xa[g][3] = x0.w;
+                        xb[g][0] = x1.x; xb[g][1] = x1.y; xb[g][2] = x1.z; xb[g][3] = x1.w;
                     }
+#pragma unroll
+                    for (int g = 0; g < NGN; ++g)
+#pragma unroll
+                        for (int bb = 0; bb < 4; ++bb)
+#pragma unroll
+                            for (int t = 0; t < TA; ++t) {
+                                acc[q][t] = fmaf(wn[g][bb][t], xa[g][bb], acc[q][t]);
+                                acc[q + 1][t] = fmaf(wn[g][bb][t], xb[g][bb], acc[q + 1][t]);
+                            }
                 }
             }
             TEAM_TT(1);
@@ -368,18 +376,23 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
                 if (i0 < npix) {
                     const float* u0 = ubase + q * qstep;
                     const float* u1 = (i0 + NPG < npix) ? u0 + qstep : u0;
+                    float xa[NGC][4], xb[NGC][4];
 #pragma unroll
                     for (int g = 0; g < NGC; ++g) {
                         const float4 x0 = *reinterpret_cast<const float4*>(u0 + offc[g]);
                         const float4 x1 = *reinterpret_cast<const float4*>(u1 + offc[g]);
-#pragma unroll
-                        for (int t = 0; t < TA; ++t) {
-                            acc[q][t] = fmaf(wc[g][0][t], x0.x, acc[q][t]); acc[q + 1][t] = fmaf(wc[g][0][t], x1.x, acc[q + 1][t]);
-                            acc[q][t] = fmaf(wc[g][1][t], x0.y, acc[q][t]); acc[q + 1][t] = fmaf(wc[g][1][t], x1.y, acc[q + 1][t]);
-                            acc[q][t] = fmaf(wc[g][2][t], x0.z, acc[q][t]); acc[q + 1][t] = fmaf(wc[g][2][t], x1.z, acc[q + 1][t]);
-                            acc[q][t] = fmaf(wc[g][3][t], x0.w, acc[q][t]); acc[q + 1][t] = fmaf(wc[g][3][t], x1.w, acc[q + 1][t]);
-                        }
+                        xa[g][0] = x0.x; xa[g][1] = x0.y; xa[g][2] = x0.z; xa[g][3] = x0.w;
+                        xb[g][0] = x1.x; xb[g][1] = x1.y; xb[g][2] = x1.z; xb[g][3] = x1.w;
                     }
+#pragma unroll
+                    for (int g = 0; g < NGC; ++g)
+#pragma unroll
+                        for (int bb = 0; bb < 4; ++bb)
+#pragma unroll
+                            for (int t = 0; t < TA; ++t) {
+                                acc[q][t] = fmaf(wc[g][bb][t], xa[g][bb], acc[q][t]);
+                                acc[q + 1][t] = fmaf(wc[g][bb][t], xb[g][bb], acc[q + 1][t]);
+                            }
                     // fold the slices that share this warp, then one partial sum per warp and pixel
                     for (int o = LG; o < 32; o <<= 1) {
 #pragma unroll
@@ -467,6 +480,282 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
 }
 
 // ---------------------------------------------------------------------------
+// Pixel-team variant: no block barrier inside a diagonal.
+//
+// A team of KW warps owns a pair of neighbouring pixels of every diagonal (and
+// further pairs NTEAM pairs apart if the diagonal is long).  The contraction
+// range is split over the KW*NS slices of the team -- over the lanes of a warp
+// first -- so each pixel's sums are folded by shuffles inside the warp, joined
+// across the team's warps through a few floats of shared memory and a named
+// barrier of the team only, and published by the team's first warp (plain
+// store + st.async to the peers, as above).  Teams never wait for one another
+// inside a step: the only cross-team dependency is the mbarrier of the
+// previous diagonal, on which one lane of every team arrives.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void named_barrier_sync(int id, int nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+template <int TA, int NGN, int NGC, int PJ>
+__global__ void __launch_bounds__(256, (NGN <= 3 ? 2 : 1)) team_pixel_kernel(TeamParams p)
+{
+    extern __shared__ __align__(128) float smem[];
+    __shared__ unsigned long long bars[2];
+    const int C = p.C, H = p.H, W = p.W, K = p.K, CS = p.CS, R = p.R, CA = p.CA;
+    const int HP = H + K - 1, WP = W + K - 1, HW = H * W;
+    const int IMG = HP * WP * CS;
+    float* U = smem;
+    float* RH = smem + IMG;
+    float* tred = smem + 2 * IMG;                   // [team][kw][2 pixels][CAp]
+    const int cl = blockIdx.x / R;
+    const int r = blockIdx.x - cl * R;
+    const int tid = threadIdx.x, NT = blockDim.x;
+    const int LG = p.LG, NS = p.NS, KW = p.KW, NTEAM = p.NPG;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int team = warp / KW, kw = warp - team * KW;
+    const int s = lane / LG, l = lane - s * LG;
+    const int gs = kw * NS + s, GSL = KW * NS;      // this thread's slice of the contraction range
+    const int CAp = LG * TA;
+    const int CB4 = (C + 3) >> 2;
+    const int GN = (K > 1 ? K * K - 2 : 1) * CB4, GC = (K > 1 ? 2 : 0) * CB4;
+    const int DS = (WP - 1) * CS;
+
+    float wn[NGN][4][TA], wc[NGC][4][TA];
+    int offn[NGN], offc[NGC];
+    auto fetch = [&](bool live, int tap, int b4, float (&dst)[4][TA], int& off) {
+        const int dh = tap / K, dw = tap - dh * K;
+        off = live ? (tap == 0 ? IMG : 0) - (dh * WP + dw) * CS + b4 * 4 : 0;
+#pragma unroll
+        for (int bb = 0; bb < 4; ++bb)
+#pragma unroll
+            for (int t = 0; t < TA; ++t) {
+                const int b = b4 * 4 + bb, al = l * TA + t;
+                float v = 0.f;
+                if (live && b < C && al < CA) v = __ldg(p.A + ((size_t)tap * C + b) * C + r * CA + al);
+                dst[bb][t] = tap == 0 ? v : -v;
+            }
+    };
+#pragma unroll
+    for (int i = 0; i < NGN; ++i) {
+        const int g = gs + i * GSL;
+        const int tnc = g / CB4, b4 = g - tnc * CB4;
+        const int tap = tnc == 0 ? 0 : (tnc <= K - 2 ? tnc + 1 : tnc + 2);
+        fetch(g < GN, g < GN ? tap : 0, b4, wn[i], offn[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < NGC; ++i) {
+        const int g = gs + i * GSL;
+        const int tcr = g / CB4, b4 = g - tcr * CB4;
+        fetch(g < GC, g < GC ? (tcr == 0 ? 1 : K) : 0, b4, wc[i], offc[i]);
+    }
+    uint32_t peerU[8], peerBar[8];
+#pragma unroll
+    for (int rr = 0; rr < 8; ++rr) {
+        const uint32_t rk = (uint32_t)(rr < R ? rr : r);
+        peerU[rr] = R > 1 ? cluster_map_u32(smem_u32(U), rk) : 0u;
+        peerBar[rr] = R > 1 ? cluster_map_u32(smem_u32(&bars[0]), rk) : 0u;
+    }
+
+    if (tid == 0) { mbar_init(&bars[0], NTEAM); mbar_init(&bars[1], NTEAM); fence_mbar_init(); }   // one arrival per team
+    for (int i = tid; i < 2 * IMG; i += NT) smem[i] = 0.f;
+    __syncthreads();
+    if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); }
+
+    const int ND = H + W - 1;
+    const int nq4 = HW >> 2;
+    unsigned stepno = 0;
+    bool alive = true;
+    for (int n = cl; n < p.B && alive; n += p.ncl) {
+        const float* src = p.rhs + (size_t)n * C * HW;
+        if (p.vec) {
+            const float4* src4 = reinterpret_cast<const float4*>(src);
+            const int nvec = C * nq4;
+            for (int v0 = tid; v0 < nvec; v0 += NT * 8) {
+                float4 tv[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (v0 + k * NT < nvec) tv[k] = __ldg(src4 + v0 + k * NT);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (v0 + k * NT < nvec) {
+                        const int vi = v0 + k * NT;
+                        const int c = fast_div(vi, p.div_q4), pp = (vi - c * nq4) << 2;
+                        const float vals[4] = {tv[k].x, tv[k].y, tv[k].z, tv[k].w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            int h = fast_div(pp + i, p.div_w), w = (pp + i) - h * W;
+                            if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
+                            RH[((h + K - 1) * WP + (w + K - 1)) * CS + c] = vals[i];
+                        }
+                    }
+                }
+            }
+        } else {
+            for (int e0 = tid; e0 < C * HW; e0 += NT * 8) {
+                float tv[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (e0 + k * NT < C * HW) tv[k] = __ldg(src + e0 + k * NT);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (e0 + k * NT < C * HW) {
+                        const int e = e0 + k * NT;
+                        const int c = fast_div(e, p.div_hw), pp = e - c * HW;
+                        int h = fast_div(pp, p.div_w), w = pp - h * W;
+                        if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
+                        RH[((h + K - 1) * WP + (w + K - 1)) * CS + c] = tv[k];
+                    }
+                }
+            }
+        }
+        __syncthreads();
+
+        for (int d = 0; d < ND; ++d, ++stepno) {
+            const int hlo = max(0, d - (W - 1));
+            const int npix = min(H - 1, d) - hlo + 1;
+            const int dbase = ((hlo + K - 1) * WP + (d - hlo) + K - 1) * CS;   // pixel 0 of the diagonal
+            float acc[PJ][2][TA];
+#pragma unroll
+            for (int j = 0; j < PJ; ++j)
+#pragma unroll
+                for (int t = 0; t < TA; ++t) { acc[j][0][t] = 0.f; acc[j][1][t] = 0.f; }
+            // taps that read diagonals <= d-2 (and the right-hand side)
+#pragma unroll
+            for (int j = 0; j < PJ; ++j) {
+                const int i0 = 2 * (team + NTEAM * j);
+                if (i0 < npix) {
+                    const float* u0 = U + dbase + i0 * DS;
+                    const float* u1 = (i0 + 1 < npix) ? u0 + DS : u0;
+#pragma unroll
+                    for (int g = 0; g < NGN; ++g) {
+                        const float4 x0 = *reinterpret_cast<const float4*>(u0 + offn[g]);
+                        const float4 x1 = *reinterpret_cast<const float4*>(u1 + offn[g]);
+                        const float a0[4] = {x0.x, x0.y, x0.z, x0.w}, a1[4] = {x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+                        for (int bb = 0; bb < 4; ++bb)
+#pragma unroll
+                            for (int t = 0; t < TA; ++t) {
+                                acc[j][0][t] = fmaf(wn[g][bb][t], a0[bb], acc[j][0][t]);
+                                acc[j][1][t] = fmaf(wn[g][bb][t], a1[bb], acc[j][1][t]);
+                            }
+                    }
+                }
+            }
+            // the previous diagonal: published by every team of this CTA and by the peers.  A single CTA uses
+            // the block barrier (every warp passes it only after its own publish of the previous step)
+            if (R == 1) {
+                __syncthreads();
+            } else if (d > 0) {
+                const unsigned prev = stepno - 1u;
+                if (!mbar_wait_bounded(&bars[prev & 1u], (prev >> 1) & 1u)) alive = false;
+            }
+            unsigned long long* mybar = &bars[stepno & 1u];
+            if (R > 1 && tid == 0) mbar_expect_tx_only(mybar, (unsigned)((R - 1) * npix * CA * 4));
+#pragma unroll
+            for (int j = 0; j < PJ; ++j) {
+                const int i0 = 2 * (team + NTEAM * j);
+                if (i0 < npix) {
+                    const bool two = i0 + 1 < npix;
+                    const float* u0 = U + dbase + i0 * DS;
+                    const float* u1 = two ? u0 + DS : u0;
+#pragma unroll
+                    for (int g = 0; g < NGC; ++g) {
+                        const float4 x0 = *reinterpret_cast<const float4*>(u0 + offc[g]);
+                        const float4 x1 = *reinterpret_cast<const float4*>(u1 + offc[g]);
+                        const float a0[4] = {x0.x, x0.y, x0.z, x0.w}, a1[4] = {x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+                        for (int bb = 0; bb < 4; ++bb)
+#pragma unroll
+                            for (int t = 0; t < TA; ++t) {
+                                acc[j][0][t] = fmaf(wc[g][bb][t], a0[bb], acc[j][0][t]);
+                                acc[j][1][t] = fmaf(wc[g][bb][t], a1[bb], acc[j][1][t]);
+                            }
+                    }
+                    // fold the slices of this warp
+                    for (int o = LG; o < 32; o <<= 1) {
+#pragma unroll
+                        for (int t = 0; t < TA; ++t) {
+                            acc[j][0][t] += __shfl_xor_sync(0xffffffffu, acc[j][0][t], o);
+                            acc[j][1][t] += __shfl_xor_sync(0xffffffffu, acc[j][1][t], o);
+                        }
+                    }
+                    if (KW > 1) {
+                        float* mine = tred + ((size_t)(team * KW + kw) * 2) * CAp + l * TA;
+                        if (kw > 0 && lane < LG) {
+#pragma unroll
+                            for (int t = 0; t < TA; ++t) { mine[t] = acc[j][0][t]; mine[CAp + t] = acc[j][1][t]; }
+                        }
+                        named_barrier_sync(1 + team, KW * 32);
+                        if (kw == 0 && lane < LG) {
+                            for (int ow = 1; ow < KW; ++ow) {
+                                const float* oth = tred + ((size_t)(team * KW + ow) * 2) * CAp + l * TA;
+#pragma unroll
+                                for (int t = 0; t < TA; ++t) { acc[j][0][t] += oth[t]; acc[j][1][t] += oth[CAp + t]; }
+                            }
+                        }
+                        if (PJ > 1) named_barrier_sync(1 + team, KW * 32);   // the next pair reuses the exchange buffer
+                    }
+                    if (kw == 0 && lane < LG) {
+                        const int o0 = dbase + i0 * DS + r * CA + l * TA;
+#pragma unroll
+                        for (int t = 0; t < TA; ++t) {
+                            if (l * TA + t < CA) {
+                                U[o0 + t] = acc[j][0][t];
+                                if (two) U[o0 + DS + t] = acc[j][1][t];
+                                if (R > 1) {
+#pragma unroll
+                                    for (int rr = 0; rr < 8; ++rr)
+                                        if (rr < R && rr != r) {
+                                            st_async_f32(peerU[rr] + 4u * (unsigned)(o0 + t), acc[j][0][t], peerBar[rr] + 8u * (stepno & 1u));
+                                            if (two)
+                                                st_async_f32(peerU[rr] + 4u * (unsigned)(o0 + DS + t), acc[j][1][t], peerBar[rr] + 8u * (stepno & 1u));
+                                        }
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            if (R > 1 && kw == 0) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(mybar);
+            }
+        }
+        if (R > 1) {
+            const unsigned prev = stepno - 1u;
+            if (!mbar_wait_bounded(&bars[prev & 1u], (prev >> 1) & 1u)) alive = false;
+        }
+        __syncthreads();
+        float* dst = p.out + (size_t)n * C * HW + (size_t)r * CA * HW;
+        if (p.vec) {
+            float4* dst4 = reinterpret_cast<float4*>(dst);
+            for (int vi = tid; vi < CA * nq4; vi += NT) {
+                const int al = fast_div(vi, p.div_q4), pp = (vi - al * nq4) << 2;
+                float vals[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    int h = fast_div(pp + i, p.div_w), w = (pp + i) - h * W;
+                    if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
+                    vals[i] = U[((h + K - 1) * WP + (w + K - 1)) * CS + r * CA + al];
+                }
+                dst4[vi] = make_float4(vals[0], vals[1], vals[2], vals[3]);
+            }
+        } else {
+            for (int e = tid; e < CA * HW; e += NT) {
+                const int al = fast_div(e, p.div_hw), pp = e - al * HW;
+                int h = fast_div(pp, p.div_w), w = pp - h * W;
+                if (p.rot) { h = H - 1 - h; w = W - 1 - w; }
+                dst[e] = U[((h + K - 1) * WP + (w + K - 1)) * CS + r * CA + al];
+            }
+        }
+        if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
+    }
+    if (!alive && tid == 0) raise_status(INVCONV_TIMEOUT);
+    if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); }
+}
+
+// ---------------------------------------------------------------------------
 // Host-side launch plan.
 // ---------------------------------------------------------------------------
 inline FastDiv make_fast_div(unsigned d)
@@ -482,15 +771,86 @@ inline FastDiv make_fast_div(unsigned d)
 
 struct TeamPlan {
     bool ok = false;
+    bool pixel = false;      // pixel-team variant
+    int KW = 1, PJ = 1;
     int R = 1, CA = 0, TA = 3, LG = 0, NS = 0, NPG = 1, CS = 0, PM = 0, NGN = 0, NGC = 0;
     int threads = 0, ncl = 0, maxt = 256;
     size_t smem = 0;
 };
 
+// Pixel-team variant: smallest estimated time over cluster size and warps per team.
+inline TeamPlan plan_team_pixel(int B, int C, int H, int W, int K, size_t max_smem, int sm_count)
+{
+    TeamPlan best;
+    double best_cost = 1e30;
+    const int CB4 = (C + 3) / 4;
+    int CS = CB4 * 4;
+    if (CS % 8 == 0) CS += 4;
+    const int GN = (K > 1 ? K * K - 2 : 1) * CB4, GC = (K > 1 ? 2 : 0) * CB4;
+    const int maxdiag = H < W ? H : W;
+    const int pairs = (maxdiag + 1) / 2;
+    const size_t img = (size_t)(H + K - 1) * (W + K - 1) * CS;
+    const int menu[3][2] = {{3, 1}, {6, 2}, {12, 3}};
+    // Measured on B200: across a cluster the slice variant is faster (wide48_k3: 108 us vs 181 us), for images
+    // that one CTA serves the pixel teams are (cifar_sq: 41 us vs 72 us); so only R = 1 is planned here unless
+    // the measurement knob asks for more.
+    const char* variant = getenv("INVCONV_TEAM_VARIANT");
+    const int rmax = (variant && variant[0] == 'p') ? 8 : 1;
+    for (int R = 1; R <= rmax; R *= 2) {
+        if (C % R != 0) continue;
+        const int CA = C / R;
+        if (R > 1 && CA < 3) continue;
+        const int TA = (CA % 3 == 0) ? 3 : 4;
+        int LG = 1;
+        while (LG * TA < CA) LG *= 2;
+        if (LG > 32) continue;
+        const int NS = 32 / LG;
+        for (int KW = 1; KW <= 4; KW *= 2) {
+            const int gsl = KW * NS;
+            const int ngn = (GN + gsl - 1) / gsl, ngc = GC > 0 ? (GC + gsl - 1) / gsl : 0;
+            int mi = -1;
+            for (int m = 0; m < 3; ++m)
+                if (ngn <= menu[m][0] && ngc <= menu[m][1]) { mi = m; break; }
+            if (mi < 0) continue;
+            int nteam = 8 / KW;
+            if (nteam > pairs) nteam = pairs;
+            const int pj = (pairs + nteam - 1) / nteam;
+            if (pj > 2) continue;
+            const size_t smem = sizeof(float) * (2 * img + (size_t)nteam * KW * 2 * LG * TA);
+            if (smem > max_smem) continue;
+            int conc = sm_count / R;                      // clusters in flight
+            if (smem * 2 + 4096 <= max_smem && menu[mi][0] <= 6) conc *= 2;   // two CTAs fit one SM
+            if (conc < 1) conc = 1;
+            const int waves = (B + conc - 1) / conc;
+            const double cost = (double)waves * pj * (menu[mi][0] + menu[mi][1] + 8 + (KW > 1 ? 4 : 0) + (R > 1 ? 4 : 0));
+            if (cost < best_cost) {
+                best_cost = cost;
+                TeamPlan pl;
+                pl.ok = true; pl.pixel = true;
+                pl.R = R; pl.CA = CA; pl.TA = TA; pl.LG = LG; pl.NS = NS; pl.CS = CS;
+                pl.NGN = menu[mi][0]; pl.NGC = menu[mi][1];
+                pl.KW = KW; pl.PJ = pj; pl.NPG = nteam; pl.PM = 0;
+                pl.threads = nteam * KW * 32;
+                pl.smem = smem;
+                int ncl = conc;
+                if (ncl > B) ncl = B;
+                pl.ncl = ncl;
+                best = pl;
+            }
+        }
+    }
+    return best;
+}
+
 inline TeamPlan plan_team(int B, int C, int H, int W, int K, size_t max_smem, int sm_count)
 {
     TeamPlan best;
     if (C < 1 || K < 1) return best;
+    const char* variant = getenv("INVCONV_TEAM_VARIANT");       // measurement knob: "slice" or "pixel"
+    if (!variant || variant[0] != 's') {
+        const TeamPlan px = plan_team_pixel(B, C, H, W, K, max_smem, sm_count);
+        if (px.ok) return px;
+    }
     // cluster size: enough CTAs that the kernel's share fits one CTA's registers, then fill the SMs
     int R = 1;
     auto divisible = [&](int rr) { return C % rr == 0 && (C / rr) >= 3; };
