@@ -54,6 +54,7 @@ constexpr size_t kMaxDynSmem = 226 * 1024;   // 227 KiB per CTA minus the kernel
 
 struct WarpPlan {
     bool ok = false;
+    bool glb = false;      // image too large for shared memory: operands stay in global memory
     int nb = 0, ipc = 0, grid = 0;
     size_t smem = 0;
 };
@@ -69,7 +70,13 @@ WarpPlan plan_warp_ck(int B, int H, int W, bool bwd)
     if (ipc > B) ipc = B > 0 ? B : 1;
     while (ipc > 1 && warp_kernel_smem<C, K>(H, W, pl.nb, ipc, bwd) > kMaxDynSmem) --ipc;
     pl.smem = warp_kernel_smem<C, K>(H, W, pl.nb, ipc, bwd);
-    if (pl.smem > kMaxDynSmem) return pl;
+    if (pl.smem > kMaxDynSmem) {
+        if (pl.nb < 2) return pl;
+        ipc = 1;
+        pl.glb = true;
+        pl.smem = warp_kernel_smem<C, K>(H, W, pl.nb, 1, bwd, true);
+        if (pl.smem > kMaxDynSmem) return pl;
+    }
     pl.ipc = ipc;
     pl.grid = (B + ipc - 1) / ipc;
     pl.ok = true;
@@ -98,7 +105,8 @@ int set_smem_limit(Kern kern, size_t smem)
 template <int C, int K, bool BWD>
 int launch_warp_ck(const WarpPlan& pl, WarpParams prm, cudaStream_t st)
 {
-    auto kern = pl.nb > 1 ? warp_wavefront_kernel<C, K, BWD, true> : warp_wavefront_kernel<C, K, BWD, false>;
+    auto kern = pl.glb ? warp_wavefront_kernel<C, K, BWD, true, true>
+                       : (pl.nb > 1 ? warp_wavefront_kernel<C, K, BWD, true> : warp_wavefront_kernel<C, K, BWD, false>);
     const int rc = set_smem_limit(kern, pl.smem);
     if (rc) return rc;
     kern<<<pl.grid, pl.nb * pl.ipc * 32, pl.smem, st>>>(prm);
@@ -119,6 +127,7 @@ int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const fl
     const bool aligned = ((reinterpret_cast<uintptr_t>(rhs) | reinterpret_cast<uintptr_t>(out) |
                            reinterpret_cast<uintptr_t>(xsaved)) & 15) == 0;
     prm.bulk = (aligned && chw % 4 == 0) ? 1 : 0;
+    prm.glb = pl.glb ? 1 : 0;
 #define X(CC, KK)                                                                         \
     if (g.C == CC && g.k == KK)                                                           \
         return bwd ? launch_warp_ck<CC, KK, true>(pl, prm, st) : launch_warp_ck<CC, KK, false>(pl, prm, st);

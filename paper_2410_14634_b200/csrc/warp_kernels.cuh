@@ -46,6 +46,7 @@ struct WarpParams {
     int nb;                // row blocks (warps) per image
     int ipc;               // images per CTA
     int bulk;              // images are 16-byte aligned multiples of 16 bytes
+    int glb;               // images stay in global memory (too large for shared memory)
 };
 
 template <int C> struct ColVec;
@@ -165,11 +166,18 @@ __device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane)
 // where grad_y[q + delta] is exactly the solved neighbour the step already
 // holds in registers; it costs one shared-memory load of x[q] and K*K*C*C FMAs
 // off the dependent chain.  The partial sums go to gw_dst[(tap*C + co)*C + ci].
-template <int C, int K, bool MULTI, bool GW>
+//
+// GLB = true serves images too large for shared memory: the right-hand side is read from, and the solution
+// written to, global memory directly (each lane walks its own row, so a 32-byte sector is fetched once and
+// then hit in L1 for eight steps; sectors are prefetched two ahead), and the K-1 bottom rows of every row
+// block go to a small shared-memory buffer `bnd` ([block][channel][row][W]) for the block below.
+template <int C, int K, bool MULTI, bool GW, bool GLB = false>
 __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int H, int W, int origin, int sgn,
                                                 int j, volatile int* progress, int lane,
-                                                const float* xs = nullptr, float* gw_dst = nullptr)
+                                                const float* xs = nullptr, float* gw_dst = nullptr,
+                                                const float* rin = nullptr, float* bnd = nullptr, int nb = 1)
 {
+    if (!GLB) rin = img;
     using S = WarpShape<C, K>;
     constexpr int KM = K - 1;
     const int HW = H * W;
@@ -208,7 +216,7 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
     int p = origin + sgn * ((32 * j + lane) * W - lane);    // offset of (lh, lw) at step 0
     float rnext[C];
 #pragma unroll
-    for (int c = 0; c < C; ++c) rnext[c] = (lane == 0 && Wl > 0) ? img[c * HW + p] : 0.f;
+    for (int c = 0; c < C; ++c) rnext[c] = (lane == 0 && Wl > 0) ? rin[c * HW + p] : 0.f;
 
     for (int s0 = 0; s0 < nsteps_up; s0 += KM) {
         if constexpr (MULTI) {
@@ -238,7 +246,16 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
             {
                 const bool act1 = (ulw + 1u) < Wl;
 #pragma unroll
-                for (int c = 0; c < C; ++c) rnext[c] = act1 ? img[c * HW + p + sgn] : 0.f;
+                for (int c = 0; c < C; ++c) rnext[c] = act1 ? rin[c * HW + p + sgn] : 0.f;
+                if constexpr (GLB) {
+                    if (((ulw + 1u) & 7u) == 0u && (ulw + 17u) < Wl) {
+#pragma unroll
+                        for (int c = 0; c < C; ++c) {
+                            asm volatile("prefetch.global.L1 [%0];" ::"l"(rin + c * HW + p + sgn * 17));
+                            if constexpr (GW) asm volatile("prefetch.global.L1 [%0];" ::"l"(xs + c * HW + p + sgn * 17));
+                        }
+                    }
+                }
             }
             // newest column of the rows above: by shuffle inside the block, from shared memory across blocks
             float nu[KM][C];
@@ -250,7 +267,10 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
                     if constexpr (MULTI) {
                         if (lane <= d) {
                             v = 0.f;
-                            if (j > 0 && active) v = img[b * HW + p - sgn * (d + 1) * W];
+                            if (j > 0 && active) {
+                                if constexpr (GLB) v = bnd[(((j - 1) * C + b) * KM + (lane - d - 1 + KM)) * W + (int)ulw];
+                                else v = img[b * HW + p - sgn * (d + 1) * W];
+                            }
                         }
                     } else if constexpr (!S::WREG) {
                         if (lane <= d) v = 0.f;
@@ -331,6 +351,12 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
             if (active) {
 #pragma unroll
                 for (int a = 0; a < C; ++a) img[a * HW + p] = acc[a];
+                if constexpr (GLB && MULTI) {
+                    if (lane >= 32 - KM && j + 1 < nb) {
+#pragma unroll
+                        for (int a = 0; a < C; ++a) bnd[((j * C + a) * KM + (lane - (32 - KM))) * W + (int)ulw] = acc[a];
+                    }
+                }
             }
             if constexpr (GW) {
 #pragma unroll
@@ -464,8 +490,10 @@ __device__ __forceinline__ void grad_w_block(const float* gy, const float* xs, i
 template <int C, int K>
 struct WarpSmem {
     using S = WarpShape<C, K>;
-    int as_off, bar_off, prog_off, red_off, img_off, imgf, total;
-    __host__ __device__ WarpSmem(int H, int W, int nb, int ipc, bool bwd)
+    int as_off, bar_off, prog_off, red_off, img_off, imgf, bnd_off, total;
+    // Hg > 0: the images stay in global memory (H = 0 is passed) and only the boundary rows between the row
+    // blocks of one image live here.
+    __host__ __device__ WarpSmem(int H, int W, int nb, int ipc, bool bwd, int Hg = 0)
     {
         auto up32 = [](int v) { return (v + 31) & ~31; };
         as_off = 0;
@@ -474,11 +502,12 @@ struct WarpSmem {
         red_off = prog_off + up32(ipc * nb);
         img_off = red_off + (bwd ? up32(nb * ipc * S::NA) : 0);
         imgf = up32(C * H * W);
-        total = img_off + imgf * ipc * (bwd ? 2 : 1);
+        bnd_off = img_off + imgf * ipc * (bwd ? 2 : 1);
+        total = bnd_off + (Hg > 0 ? up32(nb * C * (K - 1) * W) : 0);
     }
 };
 
-template <int C, int K, bool BWD, bool MULTI>
+template <int C, int K, bool BWD, bool MULTI, bool GLB = false>
 __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
 {
     using S = WarpShape<C, K>;
@@ -489,7 +518,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     const int li = warp / p.nb, j = warp - li * p.nb;  // image within the CTA, row block within the image
     const int n = blockIdx.x * p.ipc + li;             // image index
     const bool has_img = n < p.B;
-    const WarpSmem<C, K> lay(H, W, p.nb, p.ipc, BWD);
+    const WarpSmem<C, K> lay(GLB ? 0 : H, W, p.nb, p.ipc, BWD, GLB ? H : 0);
 
     float* As = smem + lay.as_off;
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + lay.bar_off);
@@ -498,12 +527,20 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     float* img = smem + lay.img_off + li * lay.imgf;                           // rhs -> solution, in place
     float* xs_all = smem + lay.img_off + p.ipc * lay.imgf;                     // backward: the saved x images
     float* xs = xs_all + li * lay.imgf;
+    float* bnd = smem + lay.bnd_off;                                           // GLB: boundary rows between row blocks
+    const float* rin = img;
+    if constexpr (GLB) {                                                        // operands stay in global memory
+        const size_t base = (size_t)(n < p.B ? n : 0) * CHW;
+        img = p.out + base;
+        rin = p.rhs + base;
+        xs = const_cast<float*>(p.xsaved ? p.xsaved + base : p.rhs + base);
+    }
 
     constexpr bool FUSE_GW = (C == 1);      // few enough partial sums to ride along in the wavefront's registers
     const bool want_gw = BWD && p.grad_w != nullptr;
     const bool leader = has_img && j == 0 && lane == 0;
     // the image's bulk copy goes out first; the kernel transform below overlaps its latency
-    if (leader && p.bulk) {
+    if (!GLB && leader && p.bulk) {
         mbar_init(&bars[li], 1);
         fence_mbar_init();
         const unsigned bytes = (unsigned)CHW * 4u;
@@ -511,7 +548,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
         bulk_g2s(img, p.rhs + (size_t)n * CHW, bytes, &bars[li]);
         if (want_gw) bulk_g2s(xs, p.xsaved + (size_t)n * CHW, bytes, &bars[li]);
     }
-    if (has_img && !p.bulk) {
+    if (!GLB && has_img && !p.bulk) {
         const float* src = p.rhs + (size_t)n * CHW;
         for (int i = j * 32 + lane; i < CHW; i += p.nb * 32) img[i] = __ldg(src + i);
         if (want_gw) {
@@ -525,21 +562,21 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
 
     bool ok = true;
     if (has_img) {
-        if (p.bulk) ok = mbar_wait_bounded(&bars[li], 0);
+        if (!GLB && p.bulk) ok = mbar_wait_bounded(&bars[li], 0);
         ok = __all_sync(0xffffffffu, ok);
         if (ok) {
             if (BWD && FUSE_GW && want_gw)
-                ok = wavefront_block<C, K, MULTI, BWD && FUSE_GW>(img, As, H, W, HW - 1, -1, j, progress + li * p.nb,
-                                                                  lane, xs, red + warp * S::NA);
+                ok = wavefront_block<C, K, MULTI, BWD && FUSE_GW, GLB>(img, As, H, W, HW - 1, -1, j, progress + li * p.nb,
+                                                                       lane, xs, red + warp * S::NA, rin, bnd, p.nb);
             else
-                ok = wavefront_block<C, K, MULTI, false>(img, As, H, W, BWD ? HW - 1 : 0, BWD ? -1 : 1, j,
-                                                         progress + li * p.nb, lane);
+                ok = wavefront_block<C, K, MULTI, false, GLB>(img, As, H, W, BWD ? HW - 1 : 0, BWD ? -1 : 1, j,
+                                                              progress + li * p.nb, lane, nullptr, nullptr, rin, bnd, p.nb);
         }
         if (!ok && lane == 0) raise_status(INVCONV_TIMEOUT);
     }
     __syncthreads();
 
-    if (has_img) {
+    if (!GLB && has_img) {
         float* dst = p.out + (size_t)n * CHW;
         if (p.bulk) {
             if (leader) {
@@ -574,7 +611,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
                 // memory of the saved-x images so that all threads have loads in flight at once.
                 __threadfence();
                 const int G = (int)gridDim.x;
-                const int chunk = min(G, (p.ipc * lay.imgf) / S::NA);
+                const int chunk = GLB ? 0 : min(G, (p.ipc * lay.imgf) / S::NA);
                 for (int b0 = 0; chunk > 0 && b0 < G; b0 += chunk) {
                     const int nbk = min(chunk, G - b0);
                     for (int idx = threadIdx.x; idx < nbk * S::NA; idx += blockDim.x)
@@ -600,13 +637,14 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
             }
         }
     }
-    if (p.bulk && leader) bulk_wait_read0();
+    if (!GLB && p.bulk && leader) bulk_wait_read0();
 }
 
 // Dynamic shared memory the kernel needs for a launch shape.
 template <int C, int K>
-inline size_t warp_kernel_smem(int H, int W, int nb, int ipc, bool bwd)
+inline size_t warp_kernel_smem(int H, int W, int nb, int ipc, bool bwd, bool glb = false)
 {
+    if (glb) return sizeof(float) * (size_t)WarpSmem<C, K>(0, W, nb, ipc, bwd, H).total;
     return sizeof(float) * (size_t)WarpSmem<C, K>(H, W, nb, ipc, bwd).total;
 }
 
