@@ -298,10 +298,8 @@ def run_ours(args, rank, world):
     ds = DeviceStep(shape, w, y, gx, device)
     sampler = ClockSampler(local)
     ms, launches = ds.time_graphs("both", args.steps, args.warmup, barrier=barrier, sampler=sampler)
-    if dist is not None:
-        t = torch.tensor([ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2410_14634_b200 import sharding
+    ms = sharding.max_over_ranks(ms, device)
     value = world * shape.B * args.steps / (ms * 1e-3)
     assert binding.invconv_get_status(device=device) == 0
 
