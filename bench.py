@@ -26,6 +26,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant (backward) kernel, one launch, from the ncu
+# capture summarised in profiles/ (per workload; None where no capture exists)
+NCU_TRAFFIC_BYTES = {"mnist": 1.633e6, "wide48_k3": None}
+
 METRIC = "invconv_fwd_bwd_images_per_sec"
 UNIT = "images/s"
 L2_BYTES = 126 * 1024 * 1024
@@ -336,7 +340,7 @@ def run_ours(args, rank, world):
                        "kernel_path": binding.invconv_path_for(shape.B, shape.C, shape.H, shape.W, shape.k)},
             "us_per_layer": {"forward": t_fwd_us, "backward": t_bwd_us, "sum": t_fwd_us + t_bwd_us},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_gbs, "unit": "GB/s",
-                         "frac": achieved / hbm_gbs, "traffic": None, "kernel": "backward (grad_y + grad_w)",
+                         "frac": achieved / hbm_gbs, "traffic": NCU_TRAFFIC_BYTES.get(args.workload), "kernel": "backward (grad_y + grad_w)",
                          "algorithmic_bytes_per_launch": dom_bytes, "peak_kind": f"of {peak_kind}"},
             "north_star_roofline": {"t_hbm_us": bd["t_hbm_us"], "t_alu_us": bd["t_alu_us"], "t_cp_us": bd["t_cp_us"],
                                     "t_step_cycles": t_step_cycles, "step_mechanism": mech, "binding": binding_name,

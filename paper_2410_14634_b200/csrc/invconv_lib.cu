@@ -612,6 +612,7 @@ int invconv_probe_step_latency(int mechanism, int steps, unsigned long long* cyc
     case 1: probe_smem_chain<<<1, 256, 0, st>>>(steps, cycles_out); break;
     case 3: probe_fma_chain<<<1, 32, 0, st>>>(steps, cycles_out); break;
     case 4: probe_group_chain<<<1, 256, 0, st>>>(steps, cycles_out); break;
+    case 5: probe_step_c3k3<<<1, 32, 0, st>>>(steps, cycles_out); break;
     case 2: {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2); cfg.blockDim = dim3(128); cfg.stream = st;

@@ -112,4 +112,62 @@ __global__ void probe_group_chain(int steps, unsigned long long* out)
     if (threadIdx.x == 0) { out[0] = (unsigned long long)(t1 - t0); out[1] = (unsigned long long)__float_as_uint(s); }
 }
 
+// Mechanism 5: the arithmetic of one wavefront step for three channels and a 3x3 kernel, registers only:
+// six shuffles, 81 FMAs on 81 per-lane weights, window rotation; no shared memory.
+__global__ void probe_step_c3k3(int steps, unsigned long long* out)
+{
+    float A[81];
+#pragma unroll
+    for (int i = 0; i < 81; ++i) A[i] = 0.001f * (i + 1) + 0.00001f * threadIdx.x;
+    float own[3][2], up[2][3][2];
+#pragma unroll
+    for (int b = 0; b < 3; ++b)
+#pragma unroll
+        for (int q = 0; q < 2; ++q) { own[b][q] = 0.1f * b + q; up[0][b][q] = 0.2f; up[1][b][q] = 0.3f; }
+    const long long t0 = clock64();
+    for (int s0 = 0; s0 < steps; s0 += 2) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            float nu[2][3];
+#pragma unroll
+            for (int d = 0; d < 2; ++d)
+#pragma unroll
+                for (int b = 0; b < 3; ++b) nu[d][b] = __shfl_up_sync(0xffffffffu, own[b][(u - 1 - d + 4) % 2], d + 1);
+            float acc[3] = {0.5f, 0.25f, 0.125f}, acc2[3] = {0.f, 0.f, 0.f};
+#pragma unroll
+            for (int dh = 0; dh < 3; ++dh)
+#pragma unroll
+                for (int dw = (dh == 0 ? 2 : 1); dw < 3; ++dw)
+#pragma unroll
+                    for (int b = 0; b < 3; ++b) {
+                        const int slot = (u - dw + 4) % 2;
+                        const float v = dh == 0 ? own[b][slot] : up[dh - 1][b][slot];
+#pragma unroll
+                        for (int a = 0; a < 3; ++a) {
+                            if ((dh * 3 + dw) & 1) acc2[a] = fmaf(-A[((dh * 3 + dw) * 3 + b) * 3 + a], v, acc2[a]);
+                            else acc[a] = fmaf(-A[((dh * 3 + dw) * 3 + b) * 3 + a], v, acc[a]);
+                        }
+                    }
+#pragma unroll
+            for (int a = 0; a < 3; ++a) acc[a] += acc2[a];
+#pragma unroll
+            for (int b = 0; b < 3; ++b)
+#pragma unroll
+                for (int a = 0; a < 3; ++a) acc[a] = fmaf(-A[(6 * 3 + b) * 3 + a], nu[1][b], acc[a]);
+#pragma unroll
+            for (int b = 0; b < 3; ++b)
+#pragma unroll
+                for (int a = 0; a < 3; ++a) acc[a] = fmaf(-A[(1 * 3 + b) * 3 + a], own[b][(u - 1 + 4) % 2], acc[a]);
+#pragma unroll
+            for (int b = 0; b < 3; ++b)
+#pragma unroll
+                for (int a = 0; a < 3; ++a) acc[a] = fmaf(-A[(3 * 3 + b) * 3 + a], nu[0][b], acc[a]);
+#pragma unroll
+            for (int b = 0; b < 3; ++b) { own[b][u] = acc[b]; up[0][b][u] = nu[0][b]; up[1][b][u] = nu[1][b]; }
+        }
+    }
+    const long long t1 = clock64();
+    if (threadIdx.x == 31) { out[0] = (unsigned long long)(t1 - t0); out[1] = (unsigned long long)__float_as_uint(own[0][0] + own[1][1] + own[2][0]); }
+}
+
 }  // namespace invconv

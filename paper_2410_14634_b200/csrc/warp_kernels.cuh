@@ -29,6 +29,8 @@
 // CTA and the last CTA to finish sums the CTA partials in a fixed order.
 #pragma once
 
+#include <cstdio>
+
 #include "common.cuh"
 #include "tma.cuh"
 
@@ -175,7 +177,8 @@ template <int C, int K, bool MULTI, bool GW, bool GLB = false>
 __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int H, int W, int origin, int sgn,
                                                 int j, volatile int* progress, int lane,
                                                 const float* xs = nullptr, float* gw_dst = nullptr,
-                                                const float* rin = nullptr, float* bnd = nullptr, int nb = 1)
+                                                const float* rin = nullptr, float* bnd = nullptr, int nb = 1,
+                                                int dummy_idx = 0)
 {
     if (!GLB) rin = img;
     using S = WarpShape<C, K>;
@@ -241,12 +244,21 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
             float xq[GW ? C : 1];
             if constexpr (GW) {
 #pragma unroll
-                for (int c = 0; c < C; ++c) xq[c] = active ? xs[c * HW + p] : 0.f;
+                for (int c = 0; c < C; ++c) {
+                    if constexpr (GLB) xq[c] = active ? xs[c * HW + p] : 0.f;
+                    else { const float t = xs[c * HW + (active ? p : origin)]; xq[c] = active ? t : 0.f; }
+                }
             }
             {
                 const bool act1 = (ulw + 1u) < Wl;
+                if constexpr (GLB) {
 #pragma unroll
-                for (int c = 0; c < C; ++c) rnext[c] = act1 ? rin[c * HW + p + sgn] : 0.f;
+                    for (int c = 0; c < C; ++c) rnext[c] = act1 ? rin[c * HW + p + sgn] : 0.f;
+                } else {
+                    const int pn = act1 ? p + sgn : origin;  // inactive lanes read a valid dummy location: no branch
+#pragma unroll
+                    for (int c = 0; c < C; ++c) { const float t = rin[c * HW + pn]; rnext[c] = act1 ? t : 0.f; }
+                }
                 if constexpr (GLB) {
                     if (((ulw + 1u) & 7u) == 0u && (ulw + 17u) < Wl) {
 #pragma unroll
@@ -265,13 +277,14 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
                 for (int b = 0; b < C; ++b) {
                     float v = __shfl_up_sync(0xffffffffu, own[b][(u - 1 - d + 2 * KM) % KM], d + 1);
                     if constexpr (MULTI) {
-                        if (lane <= d) {
-                            v = 0.f;
-                            if (j > 0 && active) {
-                                if constexpr (GLB) v = bnd[(((j - 1) * C + b) * KM + (lane - d - 1 + KM)) * W + (int)ulw];
-                                else v = img[b * HW + p - sgn * (d + 1) * W];
-                            }
-                        }
+                        // lanes whose row above lies in the previous block read it from shared memory; every lane
+                        // issues the (clamped) load so that the step stays branch-free
+                        const bool edge = lane <= d;
+                        const bool take = edge && j > 0 && active;
+                        float vb;
+                        if constexpr (GLB) vb = bnd[take ? (((j - 1) * C + b) * KM + (lane - d - 1 + KM)) * W + (int)ulw : 0];
+                        else vb = img[take ? b * HW + p - sgn * (d + 1) * W : dummy_idx];
+                        v = edge ? (take ? vb : 0.f) : v;
                     } else if constexpr (!S::WREG) {
                         if (lane <= d) v = 0.f;
                     }
@@ -348,7 +361,12 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
 #pragma unroll
                 for (int a = 0; a < C; ++a) acc[a] = fmaf(-col[a], nu[0][b], acc[a]);
             }
-            if (active) {
+            if constexpr (!GLB) {
+                // branch-free: lanes outside the image store to a scratch slot
+#pragma unroll
+                for (int a = 0; a < C; ++a) img[active ? a * HW + p : dummy_idx] = acc[a];
+            }
+            if (GLB && active) {
 #pragma unroll
                 for (int a = 0; a < C; ++a) img[a * HW + p] = acc[a];
                 if constexpr (GLB && MULTI) {
@@ -490,7 +508,7 @@ __device__ __forceinline__ void grad_w_block(const float* gy, const float* xs, i
 template <int C, int K>
 struct WarpSmem {
     using S = WarpShape<C, K>;
-    int as_off, bar_off, prog_off, red_off, img_off, imgf, bnd_off, total;
+    int as_off, bar_off, prog_off, red_off, img_off, imgf, bnd_off, dummy_off, total;
     // Hg > 0: the images stay in global memory (H = 0 is passed) and only the boundary rows between the row
     // blocks of one image live here.
     __host__ __device__ WarpSmem(int H, int W, int nb, int ipc, bool bwd, int Hg = 0)
@@ -503,7 +521,8 @@ struct WarpSmem {
         img_off = red_off + (bwd ? up32(nb * ipc * S::NA) : 0);
         imgf = up32(C * H * W);
         bnd_off = img_off + imgf * ipc * (bwd ? 2 : 1);
-        total = bnd_off + (Hg > 0 ? up32(nb * C * (K - 1) * W) : 0);
+        dummy_off = bnd_off + (Hg > 0 ? up32(nb * C * (K - 1) * W) : 0);
+        total = dummy_off + 32;
     }
 };
 
@@ -529,6 +548,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     float* xs = xs_all + li * lay.imgf;
     float* bnd = smem + lay.bnd_off;                                           // GLB: boundary rows between row blocks
     const float* rin = img;
+    const int dummy_idx = GLB ? 0 : (int)((smem + lay.dummy_off) - img);      // scratch slot for lanes outside the image
     if constexpr (GLB) {                                                        // operands stay in global memory
         const size_t base = (size_t)(n < p.B ? n : 0) * CHW;
         img = p.out + base;
@@ -536,9 +556,15 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
         xs = const_cast<float*>(p.xsaved ? p.xsaved + base : p.rhs + base);
     }
 
-    constexpr bool FUSE_GW = (C == 1);      // few enough partial sums to ride along in the wavefront's registers
+    constexpr bool FUSE_GW = (S::NA <= 81);   // few enough partial sums to ride along in the wavefront's registers
     const bool want_gw = BWD && p.grad_w != nullptr;
     const bool leader = has_img && j == 0 && lane == 0;
+#ifdef INVCONV_WARP_TIMING
+    long long tw_[6]; tw_[0] = clock64();
+#define WARP_TT(i) tw_[i] = clock64()
+#else
+#define WARP_TT(i) do { } while (0)
+#endif
     // the image's bulk copy goes out first; the kernel transform below overlaps its latency
     if (!GLB && leader && p.bulk) {
         mbar_init(&bars[li], 1);
@@ -559,21 +585,24 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     if (threadIdx.x < p.ipc * p.nb) progress[threadIdx.x] = 0;
     build_transformed_kernel<C, K, BWD>(p.w, As);
     __syncthreads();
+    WARP_TT(1);
 
     bool ok = true;
     if (has_img) {
         if (!GLB && p.bulk) ok = mbar_wait_bounded(&bars[li], 0);
         ok = __all_sync(0xffffffffu, ok);
+        WARP_TT(2);
         if (ok) {
             if (BWD && FUSE_GW && want_gw)
                 ok = wavefront_block<C, K, MULTI, BWD && FUSE_GW, GLB>(img, As, H, W, HW - 1, -1, j, progress + li * p.nb,
-                                                                       lane, xs, red + warp * S::NA, rin, bnd, p.nb);
+                                                                       lane, xs, red + warp * S::NA, rin, bnd, p.nb, dummy_idx);
             else
                 ok = wavefront_block<C, K, MULTI, false, GLB>(img, As, H, W, BWD ? HW - 1 : 0, BWD ? -1 : 1, j,
-                                                              progress + li * p.nb, lane, nullptr, nullptr, rin, bnd, p.nb);
+                                                              progress + li * p.nb, lane, nullptr, nullptr, rin, bnd, p.nb, dummy_idx);
         }
         if (!ok && lane == 0) raise_status(INVCONV_TIMEOUT);
     }
+    WARP_TT(3);
     __syncthreads();
 
     if (!GLB && has_img) {
@@ -637,7 +666,14 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
             }
         }
     }
+    WARP_TT(4);
     if (!GLB && p.bulk && leader) bulk_wait_read0();
+#ifdef INVCONV_WARP_TIMING
+    WARP_TT(5);
+    if (threadIdx.x == 0 && blockIdx.x == 0)
+        printf("warp timing (cycles): setup %lld | load wait %lld | wavefront %lld | store+gradw %lld | store drain %lld\n",
+               tw_[1] - tw_[0], tw_[2] - tw_[1], tw_[3] - tw_[2], tw_[4] - tw_[3], tw_[5] - tw_[4]);
+#endif
 }
 
 // Dynamic shared memory the kernel needs for a launch shape.
