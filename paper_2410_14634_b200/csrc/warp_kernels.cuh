@@ -221,6 +221,7 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
 #pragma unroll
     for (int c = 0; c < C; ++c) rnext[c] = (lane == 0 && Wl > 0) ? rin[c * HW + p] : 0.f;
 
+#pragma unroll 4
     for (int s0 = 0; s0 < nsteps_up; s0 += KM) {
         if constexpr (MULTI) {
             if (j > 0 && (s0 & 7) == 0) {
@@ -607,7 +608,12 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
 
     if (!GLB && has_img) {
         float* dst = p.out + (size_t)n * CHW;
-        if (p.bulk) {
+        if (p.bulk && CHW * 4 <= 16384) {
+            // small image: plain 16-byte stores retire without a completion wait at the end of the kernel
+            const float4* s4 = reinterpret_cast<const float4*>(img);
+            float4* d4 = reinterpret_cast<float4*>(dst);
+            for (int i = j * 32 + lane; i < (CHW >> 2); i += p.nb * 32) d4[i] = s4[i];
+        } else if (p.bulk) {
             if (leader) {
                 fence_proxy_async();
                 bulk_s2g(dst, img, (unsigned)CHW * 4u);
@@ -643,8 +649,16 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
                 const int chunk = GLB ? 0 : min(G, (p.ipc * lay.imgf) / S::NA);
                 for (int b0 = 0; chunk > 0 && b0 < G; b0 += chunk) {
                     const int nbk = min(chunk, G - b0);
-                    for (int idx = threadIdx.x; idx < nbk * S::NA; idx += blockDim.x)
-                        xs_all[idx] = __ldcg(p.partials + (size_t)b0 * S::NA + idx);
+                    const float* part = p.partials + (size_t)b0 * S::NA;
+                    const int tot = nbk * S::NA, nt = (int)blockDim.x;
+                    for (int i0 = threadIdx.x; i0 < tot; i0 += nt * 8) {       // eight loads in flight per thread
+                        float tv[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) tv[q] = (i0 + q * nt < tot) ? __ldcg(part + i0 + q * nt) : 0.f;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            if (i0 + q * nt < tot) xs_all[i0 + q * nt] = tv[q];
+                    }
                     __syncthreads();
                     for (int i = threadIdx.x; i < S::NA; i += blockDim.x) {
                         float s = b0 == 0 ? 0.f : red[i];
@@ -667,7 +681,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
         }
     }
     WARP_TT(4);
-    if (!GLB && p.bulk && leader) bulk_wait_read0();
+    if (!GLB && p.bulk && leader && CHW * 4 > 16384) bulk_wait_read0();
 #ifdef INVCONV_WARP_TIMING
     WARP_TT(5);
     if (threadIdx.x == 0 && blockIdx.x == 0)
