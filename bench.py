@@ -147,6 +147,9 @@ class DeviceStep:
     def fwd(self, i):
         self.b.invconv_forward(self.y[i], self.w, out=self.x[i])
 
+    def conv(self, i):
+        self.b.masked_conv_forward(self.x[i], self.w, out=self.gy[i])
+
     def bwd(self, i):
         self.b.invconv_backward(self.gx[i], self.x[i], self.w, out_grad_y=self.gy[i], out_grad_w=self.gw)
 
@@ -162,6 +165,8 @@ class DeviceStep:
                     self.fwd(i)
                 if what in ("bwd", "both"):
                     self.bwd(i)
+                if what == "conv":
+                    self.conv(i)
         launches = self.b.invconv_kernel_launch_count() - before
         self.cursor = (self.cursor + nsteps) % self.nsets
         return g, launches
@@ -378,7 +383,10 @@ def run_table(args):
         bd = bounds(shape, cyc, 1965, hbm_gbs)
         t = (ms_f + ms_b) / steps * 1e3
         roof = max(bd["t_hbm_us"], bd["t_alu_us"], bd["t_cp_us"])
+        ms_c, _ = ds.time_graphs("conv", steps, args.warmup)
         rows.append({"shape": shape.name, "path": path, "t_fwd_us": ms_f / steps * 1e3, "t_bwd_us": ms_b / steps * 1e3,
+                     "t_masked_conv_us": ms_c / steps * 1e3,
+                     "masked_conv_hbm_frac": (8.0 * shape.elements / (ms_c / steps * 1e-3) / 1e9) / hbm_gbs,
                      "images_per_s": shape.B / (t * 1e-6), **{k: bd[k] for k in ("t_hbm_us", "t_alu_us", "t_cp_us")},
                      "frac_of_roofline": roof / t})
         del ds

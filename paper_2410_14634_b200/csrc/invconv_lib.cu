@@ -15,6 +15,7 @@
 #include "warp_kernels.cuh"
 #include "team_kernels.cuh"
 #include "gradw_kernels.cuh"
+#include "conv_kernels.cuh"
 
 using namespace invconv;
 
@@ -141,6 +142,38 @@ size_t warp_workspace_bytes(int B, int C, int H, int W, int k)
     const WarpPlan pl = plan_warp(B, C, H, W, k, true);
     if (!pl.ok) return 0;
     return INVCONV_WS_CONTROL_BYTES + sizeof(float) * (size_t)pl.grid * C * C * k * k;
+}
+
+// ---------------------------------------------------------------- masked convolution, few channels
+template <int C, int K>
+int launch_masked_conv_ck(const float* x, const float* w, float* y, Geom g, cudaStream_t st)
+{
+    int wpi = (g.H + 7) / 8;                     // about eight rows per warp
+    if (wpi > 8) wpi = 8;
+    if (wpi < 1) wpi = 1;
+    int ipc = 8 / wpi;
+    if (ipc > g.B) ipc = g.B;
+    if (ipc < 1) ipc = 1;
+    while (ipc > 1 && masked_conv_smem<C, K>(g.H, g.W, ipc) > kMaxDynSmem) --ipc;
+    const size_t smem = masked_conv_smem<C, K>(g.H, g.W, ipc);
+    if (smem > kMaxDynSmem) return INVCONV_UNSUPPORTED;
+    auto kern = masked_conv_warp_kernel<C, K>;
+    const int rc = set_smem_limit(kern, smem);
+    if (rc) return rc;
+    ConvParams prm;
+    prm.x = x; prm.w = w; prm.y = y; prm.B = g.B; prm.H = g.H; prm.W = g.W; prm.ipc = ipc; prm.wpi = wpi;
+    const size_t chw = (size_t)g.C * g.H * g.W;
+    prm.bulk = ((reinterpret_cast<uintptr_t>(x) & 15) == 0 && chw % 4 == 0) ? 1 : 0;
+    kern<<<(g.B + ipc - 1) / ipc, ipc * wpi * 32, smem, st>>>(prm);
+    return check_launch();
+}
+
+int launch_masked_conv_small(const float* x, const float* w, float* y, Geom g, cudaStream_t st)
+{
+#define X(CC, KK) if (g.C == CC && g.k == KK) return launch_masked_conv_ck<CC, KK>(x, w, y, g, st);
+    INVCONV_WARP_CASES(X)
+#undef X
+    return INVCONV_UNSUPPORTED;
 }
 
 // ---------------------------------------------------------------- team family
@@ -461,6 +494,10 @@ int masked_conv_forward(const float* x, const float* w, float* y, int B, int C, 
     if (rc) return rc;
     if (B == 0) return w ? INVCONV_OK : INVCONV_BAD_ARG;
     if (!x || !w || !y || x == y) return INVCONV_BAD_ARG;
+    if (g_forced_path.load() != INVCONV_PATH_GENERIC) {
+        const int rs = launch_masked_conv_small(x, w, y, Geom{B, C, H, W, k}, as_stream(stream));
+        if (rs != INVCONV_UNSUPPORTED) return rs;
+    }
     const long long total = (long long)B * C * H * W;
     const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);
     generic_masked_conv_kernel<<<blocks, 256, 0, as_stream(stream)>>>(x, w, y, Geom{B, C, H, W, k}, total);

@@ -127,6 +127,23 @@ def test_paper_setting_unit_diagonal_one_channel(B, oracle, path):
     assert float(B.invconv_logdet(dev(w), 12, 10).item()) == 0.0
 
 
+@pytest.mark.parametrize("path", ["auto", "generic"])
+@pytest.mark.parametrize("shape", [(3, 1, 28, 28, 3), (2, 3, 32, 32, 3), (2, 3, 40, 45, 5), (1, 2, 7, 70, 2), (2, 4, 9, 9, 5),
+                                   (2, 12, 16, 16, 3), (1, 48, 8, 8, 3), (1, 3, 5, 5, 7)], ids=lambda s: "x".join(map(str, s)))
+def test_masked_conv_matches_oracle(B, oracle, shape, path):
+    """y = f(x) on its own (the sampling direction), junk in the masked-out kernel entries."""
+    import torch
+    Bn, C, H, W, k = shape
+    w, x, _ = workloads.make_custom(31 + sum(shape), Bn, C, H, W, k, sigma=0.3 / np.sqrt(C), masked_fill=float("nan"))
+    B.invconv_set_path(PATHS[path])
+    try:
+        y = B.masked_conv_forward(dev(x), dev(w))
+        torch.cuda.synchronize()
+    finally:
+        B.invconv_set_path(0)
+    assert nmax_err(y.cpu().numpy(), oracle.masked_conv(x, w)) <= 1e-5
+
+
 def test_empty_batch_is_a_no_op_and_zeroes_grad_w(B):
     import torch
     w = dev(workloads.make_custom(9, 1, 2, 4, 4, 3)[0])
