@@ -26,6 +26,7 @@
 #include <cooperative_groups.h>
 #include <cstdio>
 #include <cstdlib>
+#include <type_traits>
 
 #include "common.cuh"
 #include "tma.cuh"
@@ -179,6 +180,24 @@ struct TeamParams {
 __device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
+// Fold SPW pixel slots x TA channels across the SPW slices of a warp (slices are LG lanes apart) by halving:
+// after log2(SPW) levels the lanes of slice sw hold the warp-wide sums of pixel slot sw in v[0..TA).  This
+// takes (SPW-1)*TA shuffles where folding every value separately takes SPW*TA*log2(SPW).
+template <int SPW, int TA>
+__device__ __forceinline__ void transposed_fold(float (&v)[SPW * TA], int sw, int LG)
+{
+#pragma unroll
+    for (int hs = SPW / 2; hs >= 1; hs >>= 1) {
+        const bool hi = (sw & hs) != 0;
+#pragma unroll
+        for (int q = 0; q < hs * TA; ++q) {
+            const float send = hi ? v[q] : v[q + hs * TA];
+            const float keep = hi ? v[q + hs * TA] : v[q];
+            v[q] = keep + __shfl_xor_sync(0xffffffffu, send, hs * LG);
+        }
+    }
+}
+
 // Thread (pixel group pg, slice s, lane l) owns a few groups of four input
 // channels of one tap each and TA output channels, split into the groups whose
 // tap reads the previous diagonal (taps (0,1) and (1,0): the only ones on the
@@ -217,6 +236,7 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
     const int CB4 = (C + 3) >> 2;
     const int GN = (K > 1 ? K * K - 2 : 1) * CB4, GC = (K > 1 ? 2 : 0) * CB4;
     const int DS = (WP - 1) * CS;                   // from one pixel of a diagonal to the next (one row down, one column left)
+    const bool tfold = (LG == 4 || LG == 8 || LG == 16) && (PM % (32 / LG) == 0);   // transposed fold applies
 
     // this thread's share of the transformed kernel, signs folded in
     float wn[NGN][4][TA], wc[NGC][4][TA];
@@ -264,6 +284,9 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
     // finalize items of this thread walk (pixel, channel) pairs in steps of NT without divisions
     const int fin_i0 = tid / CA, fin_a0 = tid - fin_i0 * CA;
     const int fin_di = NT / CA, fin_da = NT - fin_di * CA;
+    const int CAQ = CA >> 2 > 0 ? CA >> 2 : 1;      // channel quads per pixel (used when CA is a multiple of four)
+    const int finq_i0 = tid / CAQ, finq_a0 = tid - finq_i0 * CAQ;
+    const int finq_di = NT / CAQ, finq_da = NT - finq_di * CAQ;
 
 #ifdef INVCONV_TEAM_TIMING
     long long tacc_[8] = {0, 0, 0, 0, 0, 0, 0, 0};
@@ -393,24 +416,53 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
                                 acc[q][t] = fmaf(wc[g][bb][t], xa[g][bb], acc[q][t]);
                                 acc[q + 1][t] = fmaf(wc[g][bb][t], xb[g][bb], acc[q + 1][t]);
                             }
-                    // fold the slices that share this warp, then one partial sum per warp and pixel
-                    for (int o = LG; o < 32; o <<= 1) {
+                    if (!tfold) {
+                        // fold the slices that share this warp, then one partial sum per warp and pixel
+                        for (int o = LG; o < 32; o <<= 1) {
 #pragma unroll
-                        for (int t = 0; t < TA; ++t) {
-                            acc[q][t] += __shfl_xor_sync(0xffffffffu, acc[q][t], o);
-                            acc[q + 1][t] += __shfl_xor_sync(0xffffffffu, acc[q + 1][t], o);
+                            for (int t = 0; t < TA; ++t) {
+                                acc[q][t] += __shfl_xor_sync(0xffffffffu, acc[q][t], o);
+                                acc[q + 1][t] += __shfl_xor_sync(0xffffffffu, acc[q + 1][t], o);
+                            }
                         }
-                    }
-                    if ((tq & 31) < LG) {
-                        float* dst = red + ((size_t)i0 * NWP + wq) * CAp + l * TA;
+                        if ((tq & 31) < LG) {
+                            float* dst = red + ((size_t)i0 * NWP + wq) * CAp + l * TA;
 #pragma unroll
-                        for (int t = 0; t < TA; ++t) dst[t] = acc[q][t];
-                        if (i0 + NPG < npix) {
+                            for (int t = 0; t < TA; ++t) dst[t] = acc[q][t];
+                            if (i0 + NPG < npix) {
 #pragma unroll
-                            for (int t = 0; t < TA; ++t) dst[NPG * NWP * CAp + t] = acc[q + 1][t];
+                                for (int t = 0; t < TA; ++t) dst[NPG * NWP * CAp + t] = acc[q + 1][t];
+                            }
                         }
                     }
                 }
+            }
+            if (tfold) {
+                // all pixel slots at once: slot sw of each round of SPW slots ends up in the lanes of slice sw
+                const int sw = (tq & 31) / LG;
+                auto fold_rounds = [&](auto spw_tag) {
+                    constexpr int SPW = decltype(spw_tag)::value;
+                    if constexpr (PM % SPW == 0) {
+#pragma unroll
+                        for (int rd = 0; rd < PM / SPW; ++rd) {
+                            if (pg + NPG * (rd * SPW) < npix) {
+                                float v[SPW * TA];
+#pragma unroll
+                                for (int x = 0; x < SPW; ++x)
+#pragma unroll
+                                    for (int t = 0; t < TA; ++t) v[x * TA + t] = acc[rd * SPW + x][t];
+                                transposed_fold<SPW, TA>(v, sw, LG);
+                                const int i = pg + NPG * (rd * SPW + sw);
+                                float* dst = red + ((size_t)i * NWP + wq) * CAp + l * TA;
+#pragma unroll
+                                for (int t = 0; t < TA; ++t) dst[t] = v[t];
+                            }
+                        }
+                    }
+                };
+                if (LG == 16) fold_rounds(std::integral_constant<int, 2>{});
+                else if (LG == 8) fold_rounds(std::integral_constant<int, 4>{});
+                else fold_rounds(std::integral_constant<int, 8>{});
             }
             TEAM_TT(3);
             __syncthreads();
@@ -419,6 +471,27 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
             unsigned long long* mybar = &bars[stepno & 1u];
             if (R > 1 && tid == 0) mbar_expect_tx_only(mybar, (unsigned)((R - 1) * npix * CA * 4));
             const int obase = ((hlo + K - 1) * WP + (d - hlo) + K - 1) * CS + r * CA;
+            if ((CA & 3) == 0) {
+                // four channels per item: one 16-byte store here and one 16-byte asynchronous store per peer
+                for (int i = finq_i0, aq = finq_a0; i < npix; ) {
+                    const float* src2 = red + (size_t)i * NWP * CAp + aq * 4;
+                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int ww = 0; ww < NWP; ++ww) {
+                        const float4 t4 = *reinterpret_cast<const float4*>(src2 + ww * CAp);
+                        v.x += t4.x; v.y += t4.y; v.z += t4.z; v.w += t4.w;
+                    }
+                    const int o = obase + i * DS + aq * 4;
+                    *reinterpret_cast<float4*>(U + o) = v;
+                    if (R > 1) {
+#pragma unroll
+                        for (int rr = 0; rr < 8; ++rr)
+                            if (rr < R && rr != r)
+                                st_async_f32x4(peerU[rr] + 4u * (unsigned)o, v, peerBar[rr] + 8u * (stepno & 1u));
+                    }
+                    i += finq_di; aq += finq_da;
+                    if (aq >= CAQ) { aq -= CAQ; ++i; }
+                }
+            } else {
             for (int i = fin_i0, al = fin_a0; i < npix; ) {
                 const float* src2 = red + (size_t)i * NWP * CAp + al;
                 float v = 0.f;
@@ -433,6 +506,7 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
                 }
                 i += fin_di; al += fin_da;
                 if (al >= CA) { al -= CA; ++i; }
+            }
             }
             __syncwarp();
             if ((tid & 31) == 0) mbar_arrive(mybar);      // the warp's stores are ordered before its one arrival
@@ -893,7 +967,7 @@ inline TeamPlan plan_team(int B, int C, int H, int W, int K, size_t max_smem, in
         pl.PM = per <= 8 ? 8 : 16;
         pl.NPG = NPG;
         pl.threads = NPG * NS * LG;
-        const size_t red = (size_t)(maxdiag + NPG) * (NS * LG / 32) * LG * TA;
+        const size_t red = (size_t)(NPG * pl.PM + NPG) * (NS * LG / 32) * LG * TA;
         pl.smem = sizeof(float) * (2 * img + red);
         if (pl.smem > max_smem) continue;
         int ncl = sm_count / R;

@@ -98,6 +98,15 @@ __device__ __forceinline__ void st_async_f32(uint32_t remote_addr, float v, uint
                  : "memory");
 }
 
+// The same for four consecutive floats (16-byte aligned).
+__device__ __forceinline__ void st_async_f32x4(uint32_t remote_addr, float4 v, uint32_t remote_bar)
+{
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.u32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(remote_addr),
+                 "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(__float_as_uint(v.z)), "r"(__float_as_uint(v.w)),
+                 "r"(remote_bar)
+                 : "memory");
+}
+
 // Division by a run-time constant through a precomputed multiplier (valid for n < 2^31).
 struct FastDiv {
     unsigned mul, shift, d;
