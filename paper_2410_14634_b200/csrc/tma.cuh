@@ -37,13 +37,16 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned 
     return done != 0;
 }
 
-// Bounded wait: gives up after a fixed number of polls (each poll may itself
-// block for a hardware-defined short time).
+// Bounded wait: polls until the phase completes or about one second of SM clock has passed (each poll may
+// itself block for a hardware-defined short time), then gives up and reports false.
 __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsigned parity)
 {
-    for (unsigned i = 0; i < (1u << 20); ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > (1ll << 31)) return false;
+    }
+    return true;
 }
 
 // global -> shared, completion counted in bytes on `bar`.
