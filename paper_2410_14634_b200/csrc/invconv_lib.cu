@@ -193,7 +193,7 @@ int sm_count()
 
 TeamPlan team_plan(int B, int C, int H, int W, int k)
 {
-    if (team_prep_smem(C) > kMaxDynSmem) return TeamPlan{};
+    if (team_solve_smem(C, k) > kMaxDynSmem) return TeamPlan{};
     return plan_team(B > 0 ? B : 1, C, H, W, k, kMaxDynSmem, sm_count());
 }
 
@@ -207,7 +207,7 @@ size_t team_workspace_bytes(int B, int C, int H, int W, int k)
     if (!team_plan(B, C, H, W, k).ok) return 0;
     const size_t na = sizeof(float) * (size_t)k * k * C * C;
     const GradWPlan gp = gradw_plan(B, C, H, W, k);
-    return INVCONV_WS_CONTROL_BYTES + na + (gp.ok ? na * gp.nbc : 0);
+    return INVCONV_WS_CONTROL_BYTES + na + sizeof(float) * (size_t)C * C + (gp.ok ? na * gp.nbc : 0);
 }
 
 template <int TC, int K>
@@ -232,7 +232,7 @@ int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, c
     const size_t na = (size_t)g.k * g.k * g.C * g.C;
     GradWParams prm;
     prm.gy = gy; prm.x = x;
-    prm.partials = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES) + na;
+    prm.partials = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES) + na + (size_t)g.C * g.C;
     prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W; prm.nbc = gp.nbc; prm.tiles = gp.tiles; prm.plane = gp.plane;
     int rc = INVCONV_UNSUPPORTED;
 #define X(TT, KK_) if (gp.TC == TT && g.k == KK_) rc = launch_gradw_inst<TT, KK_>(gp, prm, st);
@@ -299,11 +299,11 @@ int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, 
     if (!pl.ok) return INVCONV_UNSUPPORTED;
     float* A = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES);
     {
-        const size_t sm = team_prep_smem(g.C);
-        auto kern = bwd ? team_prep_kernel<true> : team_prep_kernel<false>;
+        const size_t sm = team_solve_smem(g.C, g.k);
+        auto kern = bwd ? team_solve_kernel<true> : team_solve_kernel<false>;
         const int rc = set_smem_limit(kern, sm);
         if (rc) return rc;
-        kern<<<g.k * g.k, 512, sm, st>>>(w, A, g.C, g.k);
+        kern<<<g.C + (g.C + 31) / 32, 512, sm, st>>>(w, A, g.C, g.k);
         const int rl = check_launch();
         if (rl) return rl;
     }

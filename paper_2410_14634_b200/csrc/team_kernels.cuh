@@ -4,7 +4,7 @@
 //     u[p][a] = sum_b A0[a][b] rhs[p][b] - sum_{delta != 0, b} A_delta[a][b] u[p - delta][b]
 // of length C*k^2 for each of (pixels on the diagonal) x C outputs, and the fp32
 // FMA pipe is the bound (Section 3.3: k^2 work per diagonal, here times C^2).
-// The transformed kernel A (see team_prep_kernel) is the stationary operand: it
+// The transformed kernel A (see team_solve_kernel) is the stationary operand: it
 // is distributed once over the REGISTERS of the CTA -- thread (slice s, lane l)
 // keeps the entries for its share of the contraction range (a few groups of
 // four input channels of one tap) and its TA output channels -- and stays
@@ -20,7 +20,7 @@
 //
 // The transposed solve (grad_y = M^-T grad_x, Theorem 1) runs the same kernel:
 // the image is rotated by 180 degrees while it is loaded and stored, and
-// team_prep_kernel supplies L^-T W_delta^T.
+// team_solve_kernel supplies L^-T W_delta^T.
 #pragma once
 
 #include <cooperative_groups.h>
@@ -35,7 +35,7 @@ namespace invconv {
 namespace cg = cooperative_groups;
 
 // ---------------------------------------------------------------------------
-// Transformed kernel, one CTA per tap:  A[tap][b][a], tap = dh*K + dw,
+// Transformed kernel in two steps:  A[tap][b][a], tap = dh*K + dw,
 //   forward : tap 0 -> L^-1[a][b];   tap != 0 -> sum_m L^-1[a][m] w[m][b][K-1-dh][K-1-dw]
 //   backward: tap 0 -> L^-1[b][a];   tap != 0 -> sum_m L^-1[m][a] w[b][m][K-1-dh][K-1-dw]
 // L = w[:, :, K-1, K-1] restricted to ci <= co.  L^-1 is built by blocked
@@ -44,111 +44,91 @@ namespace cg = cooperative_groups;
 // size each level, so the depth is logarithmic in C.
 // Shared memory: three C x C matrices (rows padded to 16 bytes).
 // ---------------------------------------------------------------------------
+// One CTA per input channel b (plus one for tap 0) solves  T S = RHS  by right-looking substitution in shared
+// memory, T = L (forward, rows ascending) or L^T (backward, rows descending):
+//   b <  C : RHS[m][kk] = w[m][b][kk] (forward) / w[b][m][kk] (backward); S[a][kk] -> A[flip(kk)][b][a]
+//   b >= C : RHS = 32 columns of the identity;                            S[a][b'] -> A[0][b'][a]
+// Step a scales nothing in place: every update of a later row i reads the finished row a and its diagonal,
+//   RHS[i][:] -= T[i][a] * RHS[a][:] / T[a][a],   one block barrier per row.
 template <bool BWD>
-__global__ void __launch_bounds__(512) team_prep_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K)
+__global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K)
 {
     extern __shared__ __align__(128) float sm[];
-    const int CP = (C + 3) & ~3;  // row pitch (16-byte rows)
-    float* Lm = sm;               // [C][CP] masked centre tap; later the tap's kernel slice T
-    float* Li = sm + C * CP;      // [C][CP] inverse, row-major
-    float* Sc = sm + 2 * C * CP;  // [C][CP] scratch of the merge steps; later the inverse transposed
     const int KK = K * K, ctr = KK - 1;
     const int tid = threadIdx.x, NT = blockDim.x;
-    const int tap = blockIdx.x;
-    const int dh = tap / K, dw = tap % K;
-    const int t = (K - 1 - dh) * K + (K - 1 - dw);
+    const int b = blockIdx.x;
+    const bool ident = b >= C;                // CTAs C, C+1, ...: 32-column chunks of the identity (tap 0)
+    const int c0 = ident ? (b - C) * 32 : 0;  // first identity column of this CTA
+    const int NC = ident ? min(32, C - c0) : KK;   // right-hand-side columns
+    float* L = sm;                            // [C][C]  L[i][j], j <= i
+    float* invd = sm + C * C;                 // [C]
+    float* RHS = invd + ((C + 3) & ~3);       // [C][NC]
 
-    for (int i = tid / 32; i < C; i += NT / 32)
-        for (int j = tid % 32; j < CP; j += 32) {
-            Lm[i * CP + j] = (j <= i && j < C) ? __ldg(w + (size_t)(i * C + j) * KK + ctr) : 0.f;
-            Li[i * CP + j] = 0.f;
-        }
-    __syncthreads();
-    constexpr int NB0 = 12;
-    for (int col = tid; col < C; col += NT) {       // diagonal blocks, one thread per column
-        const int o = col / NB0 * NB0, e1 = min(C, o + NB0);
-        Li[col * CP + col] = 1.0f / Lm[col * CP + col];
-        for (int i = col + 1; i < e1; ++i) {
-            float s = 0.f;
-            for (int m = col; m < i; ++m) s = fmaf(Lm[i * CP + m], Li[m * CP + col], s);
-            Li[i * CP + col] = -s / Lm[i * CP + i];
-        }
-    }
-    __syncthreads();
-    for (int sz = NB0; sz < C; sz *= 2) {
-        // every pair of neighbouring blocks (o, o+sz): X21 = -X22 * (L21 * X11)
-        const int npairs = (C + 2 * sz - 1) / (2 * sz);
-        const int per = sz * sz;
-        for (int idx = tid; idx < npairs * per; idx += NT) {
-            const int pr = idx / per, rem = idx - pr * per;
-            const int ii = rem / sz, jj = rem - ii * sz;
-            const int o = pr * 2 * sz, i = o + sz + ii, j = o + jj;
-            if (i < C) {
-                float s = 0.f;
-                for (int m = j; m < o + sz; ++m) s = fmaf(Lm[i * CP + m], Li[m * CP + j], s);
-                Sc[i * CP + j] = s;
-            }
-        }
-        __syncthreads();
-        for (int idx = tid; idx < npairs * per; idx += NT) {
-            const int pr = idx / per, rem = idx - pr * per;
-            const int ii = rem / sz, jj = rem - ii * sz;
-            const int o = pr * 2 * sz, i = o + sz + ii, j = o + jj;
-            if (i < C) {
-                float s = 0.f;
-                for (int m = o + sz; m <= i; ++m) s = fmaf(Li[i * CP + m], Sc[m * CP + j], s);
-                Li[i * CP + j] = -s;
-            }
-        }
-        __syncthreads();
-    }
-    float* out = A + (size_t)tap * C * C;
-    if (tap == 0) {
-        for (int e = tid; e < C * C; e += NT) {
-            const int b = e / C, a = e - b * C;
-            out[e] = BWD ? Li[b * CP + a] : Li[a * CP + b];
-        }
-        return;
-    }
-    // T[m][b] = w[m][b][tap]  (over Lm, which is no longer needed); the forward product wants L^-1 transposed
-    for (int i = tid / 32; i < C; i += NT / 32)
-        for (int j = tid % 32; j < CP; j += 32) {
-            Lm[i * CP + j] = j < C ? __ldg(w + (size_t)(i * C + j) * KK + t) : 0.f;
-            if (!BWD && j < C) Sc[j * CP + i] = Li[i * CP + j];
-        }
-    __syncthreads();
-    const float* T = Lm;
-    const int nq = CP / 4;
-    // thread -> (output channel a, quad of input channels b): conflict-free column reads, broadcast quads
-    for (int task = tid; task < C * nq; task += NT) {
-        const int bq = task / C, a = task - bq * C;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (!BWD) {
-            // A[b][a] = sum_{m <= a} Li[a][m] * T[m][b]
-            for (int m = 0; m <= a; ++m) {
-                const float l = Sc[m * CP + a];
-                const float4 tv = *reinterpret_cast<const float4*>(T + m * CP + bq * 4);
-                acc.x = fmaf(l, tv.x, acc.x); acc.y = fmaf(l, tv.y, acc.y);
-                acc.z = fmaf(l, tv.z, acc.z); acc.w = fmaf(l, tv.w, acc.w);
-            }
-        } else {
-            // A[b][a] = sum_{m >= a} Li[m][a] * T[b][m]
-            for (int m = a; m < C; ++m) {
-                const float l = Li[m * CP + a];
-                acc.x = fmaf(l, T[(bq * 4 + 0) * CP + m], acc.x);
-                acc.y = fmaf(l, (bq * 4 + 1 < C) ? T[(bq * 4 + 1) * CP + m] : 0.f, acc.y);
-                acc.z = fmaf(l, (bq * 4 + 2 < C) ? T[(bq * 4 + 2) * CP + m] : 0.f, acc.z);
-                acc.w = fmaf(l, (bq * 4 + 3 < C) ? T[(bq * 4 + 3) * CP + m] : 0.f, acc.w);
-            }
-        }
-        const float v[4] = {acc.x, acc.y, acc.z, acc.w};
+    for (int e0 = tid; e0 < C * C; e0 += NT * 8) {
+        float tv[8];
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-            if (bq * 4 + q < C) out[(size_t)(bq * 4 + q) * C + a] = v[q];
+        for (int q = 0; q < 8; ++q) {
+            const int e = e0 + q * NT;
+            tv[q] = (e < C * C) ? __ldg(w + (size_t)e * KK + ctr) : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int e = e0 + q * NT;
+            if (e < C * C) {
+                const int i = e / C, j = e - i * C;
+                L[e] = (j <= i) ? tv[q] : 0.f;
+                if (i == j) invd[i] = 1.0f / tv[q];
+            }
+        }
+    }
+    if (ident) {
+        for (int e = tid; e < C * NC; e += NT) RHS[e] = (e / NC == c0 + e % NC) ? 1.f : 0.f;
+    } else {
+        for (int e0 = tid; e0 < C * KK; e0 += NT * 4) {
+            float tv[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int e = e0 + q * NT;
+                if (e < C * KK) {
+                    const int m = e / KK, kk = e - m * KK;
+                    tv[q] = BWD ? __ldg(w + ((size_t)b * C + m) * KK + kk) : __ldg(w + ((size_t)m * C + b) * KK + kk);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int e = e0 + q * NT;
+                if (e < C * KK) RHS[e] = tv[q];
+            }
+        }
+    }
+    __syncthreads();
+    // thread = (row lane ty, column tx): no divisions inside the substitution loop
+    const int NCP = NC <= 32 ? 32 : NC;
+    const int tx = tid % NCP, ty = tid / NCP, TY = NT / NCP;
+    for (int st = 0; st < C - 1; ++st) {
+        const int a = BWD ? C - 1 - st : st;
+        const int nrest = C - 1 - st;                     // rows still to update
+        const float da = invd[a];
+        if (tx < NC && ty < TY) {
+            const float ra = -da * RHS[a * NC + tx];
+#pragma unroll 4
+            for (int ri = ty; ri < nrest; ri += TY) {
+                const int i = BWD ? a - 1 - ri : a + 1 + ri;
+                const float t = BWD ? L[a * C + i] : L[i * C + a];      // T[i][a]
+                RHS[i * NC + tx] = fmaf(t, ra, RHS[i * NC + tx]);
+            }
+        }
+        __syncthreads();
+    }
+    for (int e = tid; e < C * NC; e += NT) {
+        const int col = e / C, a = e - col * C;               // a fastest: coalesced stores
+        const float v = RHS[a * NC + col] * invd[a];
+        if (ident) A[(size_t)(c0 + col) * C + a] = v;         // A[0][b' = c0 + col][a]
+        else if (col != ctr) A[((size_t)(KK - 1 - col) * C + b) * C + a] = v;
     }
 }
 
-inline size_t team_prep_smem(int C) { return sizeof(float) * 3 * (size_t)C * ((C + 3) & ~3); }
+inline size_t team_solve_smem(int C, int K) { return sizeof(float) * ((size_t)C * C + ((C + 3) & ~3) + (size_t)C * (K * K > 32 ? K * K : 32)); }
 
 // ---------------------------------------------------------------------------
 struct TeamParams {
