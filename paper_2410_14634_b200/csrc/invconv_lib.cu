@@ -5,6 +5,7 @@
 
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "invconv.h"
@@ -23,6 +24,7 @@ namespace {
 
 std::atomic<int> g_forced_path{INVCONV_PATH_AUTO};
 std::atomic<unsigned long long> g_kernel_launches{0};
+std::atomic<bool> g_use_pdl{std::getenv("INVCONV_NO_PDL") == nullptr};   // measurement knob: INVCONV_NO_PDL=1 disables it
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
@@ -110,7 +112,23 @@ int launch_warp_ck(const WarpPlan& pl, WarpParams prm, cudaStream_t st)
                        : (pl.nb > 1 ? warp_wavefront_kernel<C, K, BWD, true> : warp_wavefront_kernel<C, K, BWD, false>);
     const int rc = set_smem_limit(kern, pl.smem);
     if (rc) return rc;
-    kern<<<pl.grid, pl.nb * pl.ipc * 32, pl.smem, st>>>(prm);
+    // Programmatic dependent launch: the kernel may be scheduled while its predecessor on the stream drains;
+    // it touches no global memory before griddepcontrol.wait, which waits for that predecessor to complete.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(pl.grid);
+    cfg.blockDim = dim3(pl.nb * pl.ipc * 32);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_use_pdl.load() ? 1 : 0;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
+    if (e != cudaSuccess) {
+        std::fprintf(stderr, "invconv: warp launch failed: %s\n", cudaGetErrorString(e));
+        cudaGetLastError();
+        return INVCONV_CUDA_ERROR;
+    }
     return check_launch();
 }
 

@@ -560,6 +560,11 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     constexpr bool FUSE_GW = (S::NA <= 81);   // few enough partial sums to ride along in the wavefront's registers
     const bool want_gw = BWD && p.grad_w != nullptr;
     const bool leader = has_img && j == 0 && lane == 0;
+    // everything above touched no global memory; from here on the predecessor kernel's results are needed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // let the next kernel on the stream be scheduled now; it waits at its own griddepcontrol.wait until this
+    // kernel has completed, so only its launch latency overlaps
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 #ifdef INVCONV_WARP_TIMING
     long long tw_[6]; tw_[0] = clock64();
 #define WARP_TT(i) tw_[i] = clock64()
