@@ -54,6 +54,7 @@ template <bool BWD>
 __global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K)
 {
     extern __shared__ __align__(128) float sm[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the wavefront kernel may set itself up meanwhile
     const int KK = K * K, ctr = KK - 1;
     const int tid = threadIdx.x, NT = blockDim.x;
     const int b = blockIdx.x;
@@ -218,6 +219,13 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
     const int DS = (WP - 1) * CS;                   // from one pixel of a diagonal to the next (one row down, one column left)
     const bool tfold = (LG == 4 || LG == 8 || LG == 16) && (PM % (32 / LG) == 0);   // transposed fold applies
 
+    // Set-up that needs no global memory runs first, so that under programmatic dependent launch it overlaps
+    // the kernel-transform kernel that precedes this one on the stream; griddepcontrol.wait then waits for it.
+    if (tid == 0) { mbar_init(&bars[0], NT >> 5); mbar_init(&bars[1], NT >> 5); fence_mbar_init(); }   // one arrival per warp
+    for (int i = tid; i < 2 * IMG; i += NT) smem[i] = 0.f;     // zero padding (and the channel padding) once
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     // this thread's share of the transformed kernel, signs folded in
     float wn[NGN][4][TA], wc[NGC][4][TA];
     int offn[NGN], offc[NGC];
@@ -256,8 +264,6 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
         peerBar[rr] = R > 1 ? cluster_map_u32(smem_u32(&bars[0]), rk) : 0u;
     }
 
-    if (tid == 0) { mbar_init(&bars[0], NT >> 5); mbar_init(&bars[1], NT >> 5); fence_mbar_init(); }   // one arrival per warp
-    for (int i = tid; i < 2 * IMG; i += NT) smem[i] = 0.f;     // zero padding (and the channel padding) once
     __syncthreads();
     if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); }   // every CTA's barriers exist before anyone sends
 
@@ -575,6 +581,11 @@ __global__ void __launch_bounds__(256, (NGN <= 3 ? 2 : 1)) team_pixel_kernel(Tea
     const int GN = (K > 1 ? K * K - 2 : 1) * CB4, GC = (K > 1 ? 2 : 0) * CB4;
     const int DS = (WP - 1) * CS;
 
+    if (tid == 0) { mbar_init(&bars[0], NTEAM); mbar_init(&bars[1], NTEAM); fence_mbar_init(); }   // one arrival per team
+    for (int i = tid; i < 2 * IMG; i += NT) smem[i] = 0.f;
+    asm volatile("griddepcontrol.wait;" ::: "memory");          // the kernel transform before us has completed
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     float wn[NGN][4][TA], wc[NGC][4][TA];
     int offn[NGN], offc[NGC];
     auto fetch = [&](bool live, int tap, int b4, float (&dst)[4][TA], int& off) {
@@ -611,8 +622,6 @@ __global__ void __launch_bounds__(256, (NGN <= 3 ? 2 : 1)) team_pixel_kernel(Tea
         peerBar[rr] = R > 1 ? cluster_map_u32(smem_u32(&bars[0]), rk) : 0u;
     }
 
-    if (tid == 0) { mbar_init(&bars[0], NTEAM); mbar_init(&bars[1], NTEAM); fence_mbar_init(); }   // one arrival per team
-    for (int i = tid; i < 2 * IMG; i += NT) smem[i] = 0.f;
     __syncthreads();
     if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); }
 
