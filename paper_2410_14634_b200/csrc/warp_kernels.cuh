@@ -221,7 +221,7 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
 #pragma unroll
     for (int c = 0; c < C; ++c) rnext[c] = (lane == 0 && Wl > 0) ? rin[c * HW + p] : 0.f;
 
-#pragma unroll 4
+#pragma unroll(C >= 3 ? 2 : 4)
     for (int s0 = 0; s0 < nsteps_up; s0 += KM) {
         if constexpr (MULTI) {
             if (j > 0 && (s0 & 7) == 0) {
@@ -395,7 +395,8 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
             }
 #pragma unroll
             for (int b = 0; b < C; ++b) {
-                own[b][u] = active ? acc[b] : 0.f;
+                own[b][u] = acc[b];      // lanes before their first column produce exact zeros (zero inputs), lanes past
+                                         // their last column only feed lanes that are past theirs too: no select needed
 #pragma unroll
                 for (int d = 0; d < KM; ++d) up[d][b][u] = nu[d][b];
             }
