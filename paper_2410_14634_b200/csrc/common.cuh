@@ -30,4 +30,20 @@ __host__ __device__ __forceinline__ int w_index(int co, int ci, int a, int b, in
 // Upper bound on polls of any device-side wait before it gives up.
 constexpr unsigned kMaxSpins = 1u << 22;
 
+// Sum v[0..31] over the 32 lanes; lane i returns the total of entry i.
+__device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane)
+{
+#pragma unroll
+    for (int off = 16, n = 32; off >= 1; off >>= 1, n >>= 1) {
+        const bool hi = (lane & off) != 0;
+#pragma unroll
+        for (int q = 0; q < n / 2; ++q) {
+            const float send = hi ? v[q] : v[q + n / 2];
+            const float keep = hi ? v[q + n / 2] : v[q];
+            v[q] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+    }
+    return v[0];
+}
+
 }  // namespace invconv

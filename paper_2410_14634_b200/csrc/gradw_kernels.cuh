@@ -179,4 +179,273 @@ inline GradWPlan plan_gradw(int B, int C, int H, int W, int K, size_t max_smem, 
     return pl;
 }
 
+// ---------------------------------------------------------------------------
+// Weight gradient for few channels (C <= 4): the contraction runs over B*H*W
+// pixels while there are only C*C*K*K sums, so the pixels are what is spread
+// over the GPU.  A CTA takes (image, row band) items; it stages the band's
+// grad_y rows and the x rows that reach K-1 rows above it in shared memory,
+// one bulk (TMA) copy per channel (the rows of a band are contiguous in NCHW;
+// a few large copies, because the copy engine takes on the order of a hundred
+// cycles per copy whatever its size).  A warp owns one channel pair (co, ci);
+// its lanes walk the
+// band's quads of four pixels and keep the K*K sums in registers: per quad one
+// 16-byte load of grad_y and, per kernel row, two of x and 4*K FMAs.  The
+// lanes' sums are added by shuffles, the warps' and then the CTA's sums go to
+// global memory, and the CTA that finishes last adds all CTAs' sums in CTA
+// order, negates them and applies the channel mask -- the result does not
+// depend on the order in which CTAs ran.
+// ---------------------------------------------------------------------------
+struct GradWSmallParams {
+    const float* gy;       // [B][C][H][W]
+    const float* x;        // [B][C][H][W]
+    float* partials;       // [grid][NAP]   (tap = dh*K + dw, then co, then ci)
+    float* grad_w;         // [C][C][K][K]
+    unsigned* counter;     // zero on entry; the last CTA resets it
+    int B, H, W;
+    int RB, nbands;        // rows per band, bands per image
+    int gst, xst;          // row strides of the staged grad_y and x bands (floats, multiples of 4)
+    int stage;             // floats of dynamic shared memory (the last CTA stages partial sums there)
+    int bulk;              // rows are 16-byte aligned multiples of 16 bytes: stage them with bulk copies
+    FastDiv div_bands, div_gcpr, div_xcpr, div_rb, div_xr, div_qpr;
+};
+
+template <int C, int K>
+struct GradWSmallShape {
+    static constexpr int NA = C * C * K * K, NAP = (NA + 3) & ~3, KK = K * K;
+    static constexpr int NCOMBO = C * C;                                   // channel pairs (co, ci)
+    static constexpr int WPC = C == 1 ? 16 : (C == 2 ? 4 : (C == 3 ? 2 : 1));   // warps per channel pair
+    static constexpr int NW = NCOMBO * WPC, NT = 32 * NW, NSL = 32 * WPC;
+    static_assert(KK <= 32 && NT <= 1024, "shape outside the kernel's limits");
+};
+
+template <int C, int K>
+__global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(GradWSmallParams p)
+{
+    using S = GradWSmallShape<C, K>;
+    constexpr int NA = S::NA, NAP = S::NAP, KK = S::KK, NT = S::NT, NW = S::NW, NSL = S::NSL, WPC = S::WPC;
+    extern __shared__ __align__(128) float smem[];
+    __shared__ float red[NW * KK > NA ? NW * KK : NA];
+    __shared__ unsigned long long bar;
+    __shared__ unsigned ticket;
+    const int H = p.H, W = p.W, HW = H * W, RB = p.RB, XR = RB + K - 1;
+    const int gst = p.gst, xst = p.xst;
+    float* gsm = smem;                           // [C][RB][gst]
+    float* xsm = smem + C * RB * gst;            // [C][XR][xst]
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int combo = warp / WPC, slice = (warp - combo * WPC) * 32 + lane;
+    const int co = combo / C, ci = combo - co * C;
+    const int gcpr = (gst + 31) >> 5, xcpr = (xst + 31) >> 5;      // 32-column chunks per staged row
+    const int nrow_g = C * RB;                                     // staged grad_y rows of one band
+    const int nwi_g = nrow_g * gcpr, nwi = nwi_g + C * XR * xcpr;  // (row, chunk) items of one band
+    const int qpr = gst >> 2, nq = RB * qpr;
+
+    float acc[K][K];
+#pragma unroll
+    for (int a = 0; a < K; ++a)
+#pragma unroll
+        for (int d = 0; d < K; ++d) acc[a][d] = 0.f;
+
+    // shared-memory set-up needs nothing from the predecessor kernel
+    if (tid == 0) { mbar_init(&bar, 1); fence_mbar_init(); }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#ifdef INVCONV_GW_TIMING
+    long long tg_[8]; tg_[0] = clock64(); tg_[1] = tg_[2] = tg_[5] = tg_[6] = tg_[7] = tg_[0];
+#define GW_TT(i) tg_[i] = clock64()
+#else
+#define GW_TT(i) do { } while (0)
+#endif
+    __syncthreads();
+    GW_TT(4);
+
+    unsigned phase = 0;
+    const int items = p.B * p.nbands;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int n = fast_div(item, p.div_bands), band = item - n * p.nbands;
+        const int h0 = band * RB;
+        const float* gsrc = p.gy + (size_t)n * C * HW;
+        const float* xsrc = p.x + (size_t)n * C * HW;
+        if (item != (int)blockIdx.x) __syncthreads();      // the previous band has been consumed
+        if (p.bulk) {
+            // rows outside the image are zeroed by plain stores; the rows inside arrive by one bulk copy per
+            // channel and operand (row strides equal W here, so a band is contiguous on both sides)
+            const int gv = min(RB, H - h0);                       // grad_y rows inside the image
+            const int xlo = max(0, h0 - (K - 1)), xv = min(H, h0 + RB) - xlo;   // first x row inside, and how many
+            const int xskip = xlo - (h0 - (K - 1));               // x rows above the image
+            const int gz = (RB - gv) * W, xzt = xskip * W, xzb = (XR - xskip - xv) * W;    // floats to zero per channel
+            if (gz > 0 || xzt > 0 || xzb > 0) {
+#pragma unroll 1
+                for (int c = 0; c < C; ++c) {
+                    for (int i = tid; i < gz; i += NT) gsm[(c * RB + gv) * gst + i] = 0.f;
+                    for (int i = tid; i < xzt; i += NT) xsm[c * XR * xst + i] = 0.f;
+                    for (int i = tid; i < xzb; i += NT) xsm[(c * XR + xskip + xv) * xst + i] = 0.f;
+                }
+            }
+            fence_proxy_async();
+            GW_TT(5);
+            if (warp == 0) {
+                if (lane == 0) mbar_expect_tx(&bar, (unsigned)(C * (gv + xv) * W * 4));
+                __syncwarp();
+                if (lane < C) bulk_g2s(gsm + lane * RB * gst, gsrc + lane * HW + h0 * W, (unsigned)(gv * W * 4), &bar);
+                else if (lane < 2 * C)
+                    bulk_g2s(xsm + ((lane - C) * XR + xskip) * xst, xsrc + (lane - C) * HW + xlo * W, (unsigned)(xv * W * 4), &bar);
+            }
+            GW_TT(6);
+            const bool ok = mbar_wait_bounded(&bar, phase);
+            GW_TT(7);
+            phase ^= 1u;
+            if (!__syncthreads_and(ok)) { if (tid == 0) raise_status(INVCONV_TIMEOUT); break; }
+        } else {
+            for (int wi0 = warp; wi0 < nwi; wi0 += NW * 8) {     // eight loads in flight per thread, no branches
+                float v[8];
+                int so[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int wi = wi0 + NW * q;
+                    const bool isg = wi < nwi_g;                // a grad_y row, else an x row
+                    const int wj = isg ? wi : wi - nwi_g;
+                    const int cpr = isg ? gcpr : xcpr, st = isg ? gst : xst, rows = isg ? RB : XR;
+                    const int row = isg ? fast_div(wj, p.div_gcpr) : fast_div(wj, p.div_xcpr);
+                    const int col = (wj - row * cpr) * 32 + lane;
+                    const int c = isg ? fast_div(row, p.div_rb) : fast_div(row, p.div_xr);
+                    const int h = h0 + row - c * rows - (isg ? 0 : K - 1), w = col;
+                    const bool in_s = wi < nwi && col < st;
+                    const bool in_g = in_s && w < W && h >= 0 && h < H;
+                    const float val = __ldcg((isg ? gsrc : xsrc) + (in_g ? c * HW + h * W + w : 0));
+                    v[q] = in_g ? val : 0.f;
+                    so[q] = in_s ? (isg ? 0 : C * RB * gst) + row * st + col : -1;
+                }
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (so[q] >= 0) smem[so[q]] = v[q];
+            }
+            __syncthreads();
+        }
+        GW_TT(1);
+        const float* gq = gsm + co * RB * gst;
+        const float* xq = xsm + ci * XR * xst;
+        for (int q = slice; q < nq; q += NSL) {
+            const int r = fast_div(q, p.div_qpr), w0 = (q - r * qpr) * 4;
+            const float4 g = *reinterpret_cast<const float4*>(gq + r * gst + w0);
+            const float gg[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+            for (int dh = 0; dh < K; ++dh) {
+                const float* xr = xq + (r + K - 1 - dh) * xst + w0;       // band row r meets x row r - dh
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f);               // the K-1 columns to the left of the quad
+                if (w0 > 0) a = *reinterpret_cast<const float4*>(xr - 4);
+                const float4 b = *reinterpret_cast<const float4*>(xr);
+                const float vv[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+                for (int d = 0; d < K; ++d)
+#pragma unroll
+                    for (int px = 0; px < 4; ++px) acc[dh][d] = fmaf(gg[px], vv[4 + px - d], acc[dh][d]);
+            }
+        }
+    }
+    GW_TT(2);
+
+    // lanes -> warp -> CTA
+    {
+        float v[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = i < KK ? acc[(i < KK ? i : 0) / K][(i < KK ? i : 0) % K] : 0.f;
+        const float tot = transpose_reduce32(v, lane);
+        if (lane < KK) red[warp * KK + lane] = tot;
+    }
+    __syncthreads();
+    float* part = p.partials + (size_t)blockIdx.x * NAP;
+    for (int e = tid; e < NA; e += NT) {           // e = (co*C + ci)*K*K + dh*K + dw
+        const int cb = e / KK, tap = e - cb * KK;
+        float s = 0.f;
+#pragma unroll
+        for (int sub = 0; sub < WPC; ++sub) s += red[(cb * WPC + sub) * KK + tap];
+        __stcg(part + tap * C * C + cb, s);
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) ticket = atomicAdd(p.counter, 1u);
+    __syncthreads();
+    GW_TT(3);
+#ifdef INVCONV_GW_TIMING
+    if (tid == 0 && blockIdx.x == 0)
+        printf("gradw_small (cycles) block 0: first barrier %lld | zero-fill end %lld | issued %lld | arrived %lld | last load %lld (from start) | compute end %lld | partial+ticket end %lld | ticket %u of %u\n",
+               tg_[4] - tg_[0], tg_[5] - tg_[0], tg_[6] - tg_[0], tg_[7] - tg_[0], tg_[1] - tg_[0], tg_[2] - tg_[0], tg_[3] - tg_[0], ticket, gridDim.x);
+#endif
+    if (ticket != gridDim.x - 1) return;
+
+    // last CTA: add the CTAs' sums in CTA order, staged through shared memory sixteen bytes at a time
+    __threadfence();
+    const int G = (int)gridDim.x;
+    const int chunk = min(G, p.stage / NAP);
+    for (int b0 = 0; b0 < G; b0 += chunk) {
+        const int nbk = min(chunk, G - b0);
+        const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)b0 * NAP);
+        float4* dst = reinterpret_cast<float4*>(smem);
+        const int tot4 = nbk * (NAP / 4);
+        for (int i0 = tid; i0 < tot4; i0 += NT * 8) {
+            float4 tv[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) tv[q] = __ldcg(src + min(i0 + q * NT, tot4 - 1));     // clamped: no branch
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (i0 + q * NT < tot4) dst[i0 + q * NT] = tv[q];
+        }
+        __syncthreads();
+        for (int e = tid; e < NA; e += NT) {
+            float s = b0 == 0 ? 0.f : red[e];
+#pragma unroll 8
+            for (int b = 0; b < nbk; ++b) s += smem[b * NAP + e];
+            red[e] = s;
+        }
+        __syncthreads();
+    }
+    for (int e = tid; e < NA; e += NT) {
+        const int ci_ = e % C, co_ = (e / C) % C, tap = e / (C * C);
+        const int dh_ = tap / K, dw_ = tap % K;
+        p.grad_w[((co_ * C + ci_) * K + (K - 1 - dh_)) * K + (K - 1 - dw_)] = (tap == 0 && ci_ > co_) ? 0.f : -red[e];
+    }
+    if (tid == 0) *p.counter = 0u;
+#ifdef INVCONV_GW_TIMING
+    GW_TT(4);
+    if (tid == 0) printf("gradw_small last CTA %d: total %lld | final reduce %lld\n", (int)blockIdx.x, tg_[4] - tg_[0], tg_[4] - tg_[3]);
+#endif
+}
+
+struct GradWSmallPlan {
+    bool ok = false;
+    int RB = 0, nbands = 0, gst = 0, xst = 0, grid = 0;
+    size_t smem = 0;
+};
+
+// Bands are sized so that about one CTA per SM gets an item; a band never has fewer than four rows (the K-1
+// halo rows are loaded once per band).
+inline GradWSmallPlan plan_gradw_small(int B, int C, int H, int W, int K, size_t max_smem, size_t stage_smem, int sm_count)
+{
+    GradWSmallPlan pl;
+    if (B < 1 || C > 4 || K > 5) return pl;
+    const int Wq = (W + 3) & ~3;
+    pl.gst = Wq;
+    pl.xst = Wq;
+    int nbands = sm_count / B;
+    if (nbands > (H + 3) / 4) nbands = (H + 3) / 4;
+    if (nbands < 1) nbands = 1;
+    for (;; ++nbands) {
+        const int RB = (H + nbands - 1) / nbands;
+        const size_t bytes = sizeof(float) * (size_t)C * ((size_t)RB * pl.gst + (size_t)(RB + K - 1) * pl.xst);
+        if (bytes <= max_smem) { pl.RB = RB; pl.smem = bytes; break; }
+        if (RB == 1) return pl;
+    }
+    pl.nbands = (H + pl.RB - 1) / pl.RB;
+    const int items = B * pl.nbands;
+    const int rounds = (items + sm_count - 1) / sm_count;
+    pl.grid = (items + rounds - 1) / rounds;           // every CTA takes `rounds` items (the last ones one fewer)
+    // the last CTA stages the CTAs' sums in the same shared memory: all of them at once where that fits
+    const size_t nap = (size_t)((C * C * K * K + 3) & ~3);
+    size_t want = sizeof(float) * nap * (size_t)pl.grid;
+    if (want > stage_smem) want = stage_smem - stage_smem % (sizeof(float) * nap);
+    if (pl.smem < want) pl.smem = want;
+    pl.ok = true;
+    return pl;
+}
+
 }  // namespace invconv

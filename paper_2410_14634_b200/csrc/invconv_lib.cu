@@ -132,13 +132,86 @@ int launch_warp_ck(const WarpPlan& pl, WarpParams prm, cudaStream_t st)
     return check_launch();
 }
 
+constexpr size_t kGradWSmallSmem = 96 * 1024;
+
+int sm_count();
+
+GradWSmallPlan gradw_small_plan(int B, int C, int H, int W, int k)
+{
+    return plan_gradw_small(B, C, H, W, k, kGradWSmallSmem, kMaxDynSmem - 8 * 1024, sm_count());
+}
+
+// Whether grad_w comes from the pixel-parallel kernel after the wavefront instead of riding along in it.
+// Riding along costs every diagonal step C*C*k*k extra multiply-adds on the one warp that owns the rows; the
+// separate kernel costs a launch and a second read of grad_y and x from L2.  Measured on B200, added time of
+// the separate kernel against riding along: 18 us against 10 us (C=3, 32x32, k=3, batch 128), 11 us against
+// 4 us (C=1, 28x28, k=3, batch 256), 13 us against 118 us (C=3, 64x64, k=5, batch 16, where the sums do not
+// fit the wavefront's registers), 24 us against 75 us (C=1, 256x256, k=5, batch 4, images in global memory).
+// So it is used where the sums do not fit the registers or the images stay in global memory.  INVCONV_GW_SEPARATE=0/1 overrides (measurement knob).
+bool gradw_separate(const WarpPlan& pl, const GradWSmallPlan& gs, int C, int k)
+{
+    if (!gs.ok) return false;
+    const char* knob = std::getenv("INVCONV_GW_SEPARATE");      // read per call so that tests can switch it
+    if (knob && knob[0] == '0') return false;
+    if (knob && knob[0] == '1') return true;
+    return pl.glb || C * C * k * k > 81;
+}
+
+template <int C, int K>
+int launch_gradw_small_ck(const GradWSmallPlan& gs, const GradWSmallParams& prm, cudaStream_t st)
+{
+    auto kern = gradw_small_kernel<C, K>;
+    const int rc = set_smem_limit(kern, gs.smem);
+    if (rc) return rc;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(gs.grid);
+    cfg.blockDim = dim3(GradWSmallShape<C, K>::NT);
+    cfg.dynamicSmemBytes = gs.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_use_pdl.load() ? 1 : 0;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
+    if (e != cudaSuccess) {
+        std::fprintf(stderr, "invconv: grad_w launch failed: %s\n", cudaGetErrorString(e));
+        cudaGetLastError();
+        return INVCONV_CUDA_ERROR;
+    }
+    return check_launch();
+}
+
+int launch_gradw_small(const GradWSmallPlan& gs, const float* gy, const float* x, float* gw, Geom g, void* ws, cudaStream_t st)
+{
+    GradWSmallParams prm;
+    prm.gy = gy; prm.x = x; prm.grad_w = gw;
+    prm.counter = static_cast<unsigned*>(ws);
+    prm.partials = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES);
+    prm.B = g.B; prm.H = g.H; prm.W = g.W;
+    prm.RB = gs.RB; prm.nbands = gs.nbands; prm.gst = gs.gst; prm.xst = gs.xst;
+    prm.stage = (int)(gs.smem / sizeof(float));
+    prm.bulk = (((reinterpret_cast<uintptr_t>(gy) | reinterpret_cast<uintptr_t>(x)) & 15) == 0 && g.W % 4 == 0) ? 1 : 0;
+    prm.div_bands = make_fast_div((unsigned)gs.nbands);
+    prm.div_gcpr = make_fast_div((unsigned)((gs.gst + 31) / 32));
+    prm.div_xcpr = make_fast_div((unsigned)((gs.xst + 31) / 32));
+    prm.div_rb = make_fast_div((unsigned)gs.RB);
+    prm.div_xr = make_fast_div((unsigned)(gs.RB + g.k - 1));
+    prm.div_qpr = make_fast_div((unsigned)(gs.gst / 4));
+#define X(CC, KK) if (g.C == CC && g.k == KK) return launch_gradw_small_ck<CC, KK>(gs, prm, st);
+    INVCONV_WARP_CASES(X)
+#undef X
+    return INVCONV_UNSUPPORTED;
+}
+
 int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const float* xsaved, float* gw, Geom g,
                 void* ws, cudaStream_t st)
 {
     const WarpPlan pl = plan_warp(g.B, g.C, g.H, g.W, g.k, bwd);
     if (!pl.ok) return INVCONV_UNSUPPORTED;
+    const GradWSmallPlan gs = (bwd && gw) ? gradw_small_plan(g.B, g.C, g.H, g.W, g.k) : GradWSmallPlan{};
+    const bool separate = bwd && gw && ws && gradw_separate(pl, gs, g.C, g.k);
     WarpParams prm;
-    prm.rhs = rhs; prm.w = w; prm.out = out; prm.xsaved = xsaved; prm.grad_w = gw;
+    prm.rhs = rhs; prm.w = w; prm.out = out; prm.xsaved = xsaved; prm.grad_w = separate ? nullptr : gw;
     prm.counter = static_cast<unsigned*>(ws);
     prm.partials = ws ? reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES) : nullptr;
     prm.B = g.B; prm.H = g.H; prm.W = g.W; prm.nb = pl.nb; prm.ipc = pl.ipc;
@@ -147,19 +220,25 @@ int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const fl
                            reinterpret_cast<uintptr_t>(xsaved)) & 15) == 0;
     prm.bulk = (aligned && chw % 4 == 0) ? 1 : 0;
     prm.glb = pl.glb ? 1 : 0;
+    int rc = INVCONV_UNSUPPORTED;
 #define X(CC, KK)                                                                         \
     if (g.C == CC && g.k == KK)                                                           \
-        return bwd ? launch_warp_ck<CC, KK, true>(pl, prm, st) : launch_warp_ck<CC, KK, false>(pl, prm, st);
+        rc = bwd ? launch_warp_ck<CC, KK, true>(pl, prm, st) : launch_warp_ck<CC, KK, false>(pl, prm, st);
     INVCONV_WARP_CASES(X)
 #undef X
-    return INVCONV_UNSUPPORTED;
+    if (rc || !separate) return rc;
+    return launch_gradw_small(gs, out, xsaved, gw, g, ws, st);
 }
 
 size_t warp_workspace_bytes(int B, int C, int H, int W, int k)
 {
     const WarpPlan pl = plan_warp(B, C, H, W, k, true);
     if (!pl.ok) return 0;
-    return INVCONV_WS_CONTROL_BYTES + sizeof(float) * (size_t)pl.grid * C * C * k * k;
+    const size_t na = (size_t)C * C * k * k;
+    size_t floats = (size_t)pl.grid * na;
+    const GradWSmallPlan gs = gradw_small_plan(B > 0 ? B : 1, C, H, W, k);
+    if (gs.ok && (size_t)gs.grid * ((na + 3) & ~(size_t)3) > floats) floats = (size_t)gs.grid * ((na + 3) & ~(size_t)3);
+    return INVCONV_WS_CONTROL_BYTES + sizeof(float) * floats;
 }
 
 // ---------------------------------------------------------------- masked convolution, few channels

@@ -821,17 +821,6 @@ __global__ void __launch_bounds__(256, (NGN <= 3 ? 2 : 1)) team_pixel_kernel(Tea
 // ---------------------------------------------------------------------------
 // Host-side launch plan.
 // ---------------------------------------------------------------------------
-inline FastDiv make_fast_div(unsigned d)
-{
-    FastDiv f;
-    f.d = d;
-    unsigned sh = 0;
-    while ((1ull << sh) < d) ++sh;
-    f.shift = sh;
-    f.mul = (unsigned)((((1ull << sh) - d) << 32) / d + 1);
-    return f;
-}
-
 struct TeamPlan {
     bool ok = false;
     bool pixel = false;      // pixel-team variant

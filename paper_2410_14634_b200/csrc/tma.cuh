@@ -119,4 +119,17 @@ __device__ __forceinline__ int fast_div(int n, FastDiv f)
     return (int)((__umulhi((unsigned)n, f.mul) + (unsigned)n) >> f.shift);
 }
 
+
+// Host side: the multiplier and shift for fast_div by d >= 1.
+inline FastDiv make_fast_div(unsigned d)
+{
+    FastDiv f;
+    f.d = d;
+    unsigned sh = 0;
+    while ((1ull << sh) < d) ++sh;
+    f.shift = sh;
+    f.mul = (unsigned)((((1ull << sh) - d) << 32) / d + 1);
+    return f;
+}
+
 }  // namespace invconv

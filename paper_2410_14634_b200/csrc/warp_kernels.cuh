@@ -135,22 +135,6 @@ __device__ void build_transformed_kernel(const float* __restrict__ w, float* As)
     }
 }
 
-// Sum v[0..31] over the 32 lanes; lane i returns the total of entry i.
-__device__ __forceinline__ float transpose_reduce32(float (&v)[32], int lane)
-{
-#pragma unroll
-    for (int off = 16, n = 32; off >= 1; off >>= 1, n >>= 1) {
-        const bool hi = (lane & off) != 0;
-#pragma unroll
-        for (int q = 0; q < n / 2; ++q) {
-            const float send = hi ? v[q] : v[q + n / 2];
-            const float keep = hi ? v[q + n / 2] : v[q];
-            v[q] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-        }
-    }
-    return v[0];
-}
-
 // The wavefront over one block of up to 32 rows.  Logical pixel (lh, lw) of
 // channel c lives at img[c*HW + origin + sgn*(lh*W + lw)] (sgn = -1 walks the
 // rotated image of the transposed solve).  Returns false if a wait gave up.

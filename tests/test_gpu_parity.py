@@ -111,6 +111,53 @@ def test_edge_shapes(B, oracle, shape, path):
     check_all(B, oracle, w, y, gx, path)
 
 
+GW_SEPARATE = [  # shapes for the pixel-parallel grad_w kernel: ragged widths, bands with and without halo rows,
+    # more (image, band) items than CTAs, a single pixel, every (C, k) the few-channel family serves
+    (1, 1, 1, 1, 2), (3, 1, 28, 28, 3), (2, 3, 32, 32, 3), (1, 3, 64, 64, 5), (2, 4, 9, 11, 5), (1, 2, 7, 9, 5),
+    (170, 1, 8, 8, 3), (300, 2, 4, 4, 2), (1, 4, 40, 36, 3), (2, 3, 33, 30, 2), (1, 1, 130, 260, 5), (5, 4, 16, 16, 5),
+]
+
+
+@pytest.mark.parametrize("separate", ["0", "1"])
+@pytest.mark.parametrize("shape", GW_SEPARATE, ids=lambda s: "x".join(map(str, s)))
+def test_grad_w_inside_or_after_the_wavefront(B, oracle, shape, separate, monkeypatch):
+    """Both ways of computing grad_w on the few-channel path (riding along in the wavefront kernel, or the
+    pixel-parallel kernel after it) against the oracle, and twice in a row (the ticket counter is reset)."""
+    monkeypatch.setenv("INVCONV_GW_SEPARATE", separate)
+    Bn, C, H, W, k = shape
+    w, y, gx = workloads.make_custom(300 + sum(shape), Bn, C, H, W, k, sigma=0.05 / np.sqrt(C))
+    check_all(B, oracle, w, y, gx, "warp")
+    check_all(B, oracle, w, y, gx, "warp")
+
+
+def test_grad_w_after_the_wavefront_with_unaligned_buffers(B, oracle, monkeypatch):
+    """Buffers that start 4 bytes off a 16-byte boundary take the plain-load staging path."""
+    import torch
+    monkeypatch.setenv("INVCONV_GW_SEPARATE", "1")
+    Bn, C, H, W, k = 3, 3, 12, 16, 3
+    w, y, gx = workloads.make_custom(77, Bn, C, H, W, k)
+    n = y.size
+    def off(a):
+        buf = torch.empty(n + 1, dtype=torch.float32, device="cuda")
+        v = buf[1:].view(a.shape)
+        v.copy_(torch.from_numpy(a))
+        return v
+    B.invconv_set_path(PATHS["warp"])
+    try:
+        x = B.invconv_forward(off(y), dev(w))
+        gy = torch.empty(n + 1, dtype=torch.float32, device="cuda")[1:].view(y.shape)
+        _, gw = B.invconv_backward(off(gx), off(x.cpu().numpy()), dev(w), out_grad_y=gy)
+        torch.cuda.synchronize()
+        assert B.invconv_get_status() == 0
+    finally:
+        B.invconv_set_path(0)
+    x64 = x.cpu().numpy().astype(np.float64)
+    gy_ref = oracle.invconv_grad_y(gx, w)
+    gw_ref = oracle.invconv_grad_w(gy_ref, x64, w.shape[-1])
+    assert nmax_err(gy.cpu().numpy(), gy_ref) <= 1e-4
+    assert nmax_err(gw.cpu().numpy(), gw_ref) <= 1e-3
+
+
 @pytest.mark.parametrize("path", ["auto", "generic", "warp", "team"])
 def test_masked_out_kernel_entries_are_never_read(B, oracle, path):
     for (Bn, C, H, W, k) in [(2, 3, 9, 8, 3), (1, 12, 6, 6, 3)]:
