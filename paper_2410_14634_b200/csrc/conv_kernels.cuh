@@ -137,4 +137,201 @@ inline size_t masked_conv_smem(int H, int W, int ipc)
     return sizeof(float) * ((((size_t)C * C * K * K + 31) & ~(size_t)31) + 32 + imgf * ipc);
 }
 
+// ---------------------------------------------------------------------------
+// y = f(x) for many channels: a dense contraction over (ci, dh, dw) with
+// C*K*K multiply-adds per output element, bound by the fp32 FMA pipe.
+//
+// A CTA owns 16 output channels and up to 64 quads of four horizontally
+// adjacent pixels (a band of rows of one image, or several small images).  A
+// thread owns one quad and four output channels: 16 sums in registers.  The
+// input channels arrive eight at a time, double-buffered with asynchronous
+// copies: the x rows of the band (plus the K-1 rows above it; every staged row
+// carries four zero columns on its left so that the K-1 pixels to the left of
+// a quad come with the aligned quad before it) and the CTA's slice of the
+// kernel, re-ordered to [ci][dh][co group][dw][co] with the channel mask of
+// the bottom-right tap applied.  Per (ci, dh) a thread issues two 16-byte
+// loads of x and K 16-byte broadcast loads of the kernel for 16*K FMAs.
+// ---------------------------------------------------------------------------
+struct ConvTileParams {
+    const float* x;
+    const float* w;
+    float* y;
+    int B, C, H, W;
+    int RB, nbands;        // rows per band, bands per image
+    int Q, IPC;            // quads per band, bands (items) per CTA
+    int PW, PH;            // floats per staged row (4 + W rounded up to 4), staged rows per band (RB + K - 1)
+    int cotiles;           // tiles of 16 output channels
+    int vec;               // x and y are 16-byte aligned and W % 4 == 0
+    FastDiv div_q, div_qpr, div_bands, div_ph;
+};
+
+constexpr int kConvCoT = 16, kConvCiT = 8;
+
+template <int K>
+__global__ void __launch_bounds__(256) masked_conv_tile_kernel(ConvTileParams p)
+{
+    constexpr int CO_T = kConvCoT, CI_T = kConvCiT, KK = K * K;
+    constexpr int WBUF = CI_T * K * 4 * K * 4;          // floats of one kernel buffer: [ci][dh][cg][dw][4]
+    extern __shared__ __align__(128) float smem[];
+    const int C = p.C, H = p.H, W = p.W, PW = p.PW, PH = p.PH, RB = p.RB;
+    const int plane = PH * PW;                           // one staged channel of one band
+    const int XBUF = p.IPC * CI_T * plane;
+    float* xsm = smem;                                   // [2][IPC][CI_T][PH][PW]
+    float* wsm = smem + 2 * XBUF;                        // [2][WBUF]
+    const int tid = threadIdx.x, NT = blockDim.x, SL = NT >> 2;
+    const int cg = tid / SL, slot = tid - cg * SL;       // warps are uniform in cg (SL is a multiple of 32)
+    const int cot = blockIdx.x % p.cotiles, group = blockIdx.x / p.cotiles;
+    const int co0 = cot * CO_T;
+    const int nitems = p.B * p.nbands;
+    const int qpr = (PW - 4) >> 2;
+
+    // this thread's quad
+    const int li = fast_div(slot, p.div_q), q = slot - li * p.Q;
+    const int r = fast_div(q, p.div_qpr), w0 = (q - r * qpr) * 4;
+    const int item = group * p.IPC + li;
+    const bool has_quad = li < p.IPC && item < nitems;
+    const int n_img = fast_div(item, p.div_bands), band = item - n_img * p.nbands;
+    const int h = band * RB + r;
+
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    // the four zero columns on the left of every staged row (never overwritten)
+    for (int i = tid; i < 2 * p.IPC * CI_T * PH; i += NT) *reinterpret_cast<float4*>(xsm + i * PW) = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    auto stage = [&](int chunk, int buf) {
+        const int ci0 = chunk * CI_T;
+        // kernel slice: source order (co, ci, a, b) so that consecutive threads read consecutive floats
+        float* wb = wsm + buf * WBUF;
+        for (int e = tid; e < CO_T * CI_T * KK; e += NT) {
+            const int col = e / (CI_T * KK), rem = e - col * (CI_T * KK);
+            const int cil = rem / KK, ab = rem - cil * KK, a = ab / K, b = ab - a * K;
+            const int co = co0 + col, ci = ci0 + cil, dh = K - 1 - a, dw = K - 1 - b;
+            const bool valid = co < C && ci < C && !(ab == KK - 1 && ci > co);
+            const float* src = p.w + (valid ? ((size_t)(co * C + ci) * KK + ab) : 0);
+            cp_async_f32(wb + (((cil * K + dh) * 4 + (col >> 2)) * K + dw) * 4 + (col & 3), src, valid);
+        }
+        // x rows of the band and the K-1 rows above it
+        float* xb = xsm + buf * XBUF;
+        if (p.vec) {
+            const int per_item = CI_T * PH * qpr;
+            for (int e = tid; e < p.IPC * per_item; e += NT) {
+                const int l = e / per_item, rem = e - l * per_item;       // IPC and CI_T*PH*qpr are small: plain division
+                const int row = fast_div(rem, p.div_qpr), qx = rem - row * qpr;
+                const int cil = fast_div(row, p.div_ph), rr = row - cil * PH;
+                const int it = group * p.IPC + l;
+                const int n = fast_div(it, p.div_bands), bd = it - n * p.nbands;
+                const int hh = bd * RB - (K - 1) + rr, ci = ci0 + cil;
+                const bool valid = it < nitems && ci < C && hh >= 0 && hh < H;
+                const float* src = p.x + (valid ? (((size_t)n * C + ci) * H + hh) * W + 4 * qx : 0);
+                cp_async_f32x4(xb + (l * CI_T + cil) * plane + rr * PW + 4 + 4 * qx, src, valid);
+            }
+        } else {
+            const int per_item = CI_T * PH * (PW - 4);
+            for (int e = tid; e < p.IPC * per_item; e += NT) {
+                const int l = e / per_item, rem = e - l * per_item;
+                const int row = rem / (PW - 4), cx = rem - row * (PW - 4);
+                const int cil = fast_div(row, p.div_ph), rr = row - cil * PH;
+                const int it = group * p.IPC + l;
+                const int n = fast_div(it, p.div_bands), bd = it - n * p.nbands;
+                const int hh = bd * RB - (K - 1) + rr, ci = ci0 + cil;
+                const bool valid = it < nitems && ci < C && hh >= 0 && hh < H && cx < W;
+                const float* src = p.x + (valid ? (((size_t)n * C + ci) * H + hh) * W + cx : 0);
+                cp_async_f32(xb + (l * CI_T + cil) * plane + rr * PW + 4 + cx, src, valid);
+            }
+        }
+        cp_async_commit();
+    };
+
+    const int nchunks = (C + CI_T - 1) / CI_T;
+    stage(0, 0);
+    for (int chunk = 0; chunk < nchunks; ++chunk) {
+        const int buf = chunk & 1;
+        if (chunk + 1 < nchunks) { stage(chunk + 1, buf ^ 1); cp_async_wait<1>(); }
+        else cp_async_wait<0>();
+        __syncthreads();
+        if (has_quad) {
+            const float* xq = xsm + buf * XBUF + li * CI_T * plane + r * PW + w0;     // row r of the band is staged row r + K-1
+            const float* wq = wsm + buf * WBUF + cg * K * 4;
+#pragma unroll 2
+            for (int cil = 0; cil < CI_T; ++cil) {
+#pragma unroll
+                for (int dh = 0; dh < K; ++dh) {
+                    const float* xr = xq + cil * plane + (K - 1 - dh) * PW;
+                    const float4 a = *reinterpret_cast<const float4*>(xr);
+                    const float4 b = *reinterpret_cast<const float4*>(xr + 4);
+                    const float vv[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+                    for (int dw = 0; dw < K; ++dw) {
+                        const float4 wv = *reinterpret_cast<const float4*>(wq + ((cil * K + dh) * 4 * K + dw) * 4);
+#pragma unroll
+                        for (int px = 0; px < 4; ++px) {
+                            const float v = vv[4 + px - dw];
+                            acc[px][0] = fmaf(v, wv.x, acc[px][0]);
+                            acc[px][1] = fmaf(v, wv.y, acc[px][1]);
+                            acc[px][2] = fmaf(v, wv.z, acc[px][2]);
+                            acc[px][3] = fmaf(v, wv.w, acc[px][3]);
+                        }
+                    }
+                }
+            }
+        }
+        __syncthreads();       // the buffer is free for the copies of chunk + 2
+    }
+
+    if (has_quad && h < H) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int co = co0 + cg * 4 + j;
+            if (co < C) {
+                float* dst = p.y + (((size_t)n_img * C + co) * H + h) * W + w0;
+                if (p.vec) *reinterpret_cast<float4*>(dst) = make_float4(acc[0][j], acc[1][j], acc[2][j], acc[3][j]);
+                else {
+#pragma unroll
+                    for (int px = 0; px < 4; ++px)
+                        if (w0 + px < W) dst[px] = acc[px][j];
+                }
+            }
+        }
+    }
+}
+
+struct ConvTilePlan {
+    bool ok = false;
+    int RB = 0, nbands = 0, Q = 0, IPC = 1, PW = 0, PH = 0, cotiles = 0, threads = 0, grid = 0;
+    size_t smem = 0;
+};
+
+inline ConvTilePlan plan_conv_tile(int B, int C, int H, int W, int K, size_t max_smem, int sm_count)
+{
+    ConvTilePlan pl;
+    if (B < 1 || K > 5 || C < 5) return pl;
+    const int qpr = (W + 3) / 4;
+    if (qpr > 64) return pl;
+    pl.PW = 4 + 4 * qpr;
+    pl.RB = 64 / qpr;
+    if (pl.RB > H) pl.RB = H;
+    pl.nbands = (H + pl.RB - 1) / pl.RB;
+    pl.RB = (H + pl.nbands - 1) / pl.nbands;            // even bands
+    pl.Q = pl.RB * qpr;
+    pl.PH = pl.RB + K - 1;
+    pl.cotiles = (C + kConvCoT - 1) / kConvCoT;
+    const int items = B * pl.nbands;
+    int ipc = 64 / pl.Q;
+    if (ipc < 1) ipc = 1;
+    const int ipc_min = pl.Q >= 32 ? 1 : (32 + pl.Q - 1) / pl.Q;       // fill at least one warp per output-channel group
+    while (ipc > ipc_min && ((items + ipc - 1) / ipc) * pl.cotiles < 2 * sm_count) --ipc;   // enough CTAs first
+    pl.IPC = ipc;
+    const int slots = (ipc * pl.Q + 31) & ~31;
+    pl.threads = 4 * slots;
+    pl.smem = sizeof(float) * 2 * ((size_t)ipc * kConvCiT * pl.PH * pl.PW + (size_t)kConvCiT * K * 4 * K * 4);
+    if (pl.threads > 256 || pl.smem > max_smem) return pl;
+    pl.grid = ((items + ipc - 1) / ipc) * pl.cotiles;
+    pl.ok = true;
+    return pl;
+}
+
 }  // namespace invconv

@@ -265,6 +265,40 @@ int launch_masked_conv_ck(const float* x, const float* w, float* y, Geom g, cuda
     return check_launch();
 }
 
+template <int K>
+int launch_masked_conv_tile_k(const ConvTilePlan& pl, const ConvTileParams& prm, cudaStream_t st)
+{
+    auto kern = masked_conv_tile_kernel<K>;
+    const int rc = set_smem_limit(kern, pl.smem);
+    if (rc) return rc;
+    kern<<<pl.grid, pl.threads, pl.smem, st>>>(prm);
+    return check_launch();
+}
+
+// Many channels: the register-tiled kernel; INVCONV_UNSUPPORTED where its plan does not fit.
+int launch_masked_conv_tile(const float* x, const float* w, float* y, Geom g, cudaStream_t st)
+{
+    const ConvTilePlan pl = plan_conv_tile(g.B, g.C, g.H, g.W, g.k, kMaxDynSmem / 2, sm_count());
+    if (!pl.ok) return INVCONV_UNSUPPORTED;
+    ConvTileParams prm;
+    prm.x = x; prm.w = w; prm.y = y; prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W;
+    prm.RB = pl.RB; prm.nbands = pl.nbands; prm.Q = pl.Q; prm.IPC = pl.IPC; prm.PW = pl.PW; prm.PH = pl.PH;
+    prm.cotiles = pl.cotiles;
+    prm.vec = (((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15) == 0 && g.W % 4 == 0) ? 1 : 0;
+    prm.div_q = make_fast_div((unsigned)pl.Q);
+    prm.div_qpr = make_fast_div((unsigned)((pl.PW - 4) / 4));
+    prm.div_bands = make_fast_div((unsigned)pl.nbands);
+    prm.div_ph = make_fast_div((unsigned)pl.PH);
+    switch (g.k) {
+    case 1: return launch_masked_conv_tile_k<1>(pl, prm, st);
+    case 2: return launch_masked_conv_tile_k<2>(pl, prm, st);
+    case 3: return launch_masked_conv_tile_k<3>(pl, prm, st);
+    case 4: return launch_masked_conv_tile_k<4>(pl, prm, st);
+    case 5: return launch_masked_conv_tile_k<5>(pl, prm, st);
+    default: return INVCONV_UNSUPPORTED;
+    }
+}
+
 int launch_masked_conv_small(const float* x, const float* w, float* y, Geom g, cudaStream_t st)
 {
 #define X(CC, KK) if (g.C == CC && g.k == KK) return launch_masked_conv_ck<CC, KK>(x, w, y, g, st);
@@ -598,6 +632,8 @@ int masked_conv_forward(const float* x, const float* w, float* y, int B, int C, 
     if (g_forced_path.load() != INVCONV_PATH_GENERIC) {
         const int rs = launch_masked_conv_small(x, w, y, Geom{B, C, H, W, k}, as_stream(stream));
         if (rs != INVCONV_UNSUPPORTED) return rs;
+        const int rt = launch_masked_conv_tile(x, w, y, Geom{B, C, H, W, k}, as_stream(stream));
+        if (rt != INVCONV_UNSUPPORTED) return rt;
     }
     const long long total = (long long)B * C * H * W;
     const int blocks = (int)((total + 255) / 256 < 148LL * 16 ? (total + 255) / 256 : 148LL * 16);

@@ -110,6 +110,20 @@ __device__ __forceinline__ void st_async_f32x4(uint32_t remote_addr, float4 v, u
                  : "memory");
 }
 
+// Asynchronous global -> shared copies of 4 and 16 bytes (LDGSTS); `valid == false` writes zeros and reads
+// nothing (the source address must still be a mapped one).
+__device__ __forceinline__ void cp_async_f32(float* dst_smem, const float* src, bool valid)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst_smem)), "l"(src), "r"(valid ? 4 : 0) : "memory");
+}
+__device__ __forceinline__ void cp_async_f32x4(float* dst_smem, const float* src, bool valid)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst_smem)), "l"(src), "r"(valid ? 16 : 0) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // Division by a run-time constant through a precomputed multiplier (valid for n < 2^31).
 struct FastDiv {
     unsigned mul, shift, d;

@@ -176,7 +176,12 @@ def test_paper_setting_unit_diagonal_one_channel(B, oracle, path):
 
 @pytest.mark.parametrize("path", ["auto", "generic"])
 @pytest.mark.parametrize("shape", [(3, 1, 28, 28, 3), (2, 3, 32, 32, 3), (2, 3, 40, 45, 5), (1, 2, 7, 70, 2), (2, 4, 9, 9, 5),
-                                   (2, 12, 16, 16, 3), (1, 48, 8, 8, 3), (1, 3, 5, 5, 7)], ids=lambda s: "x".join(map(str, s)))
+                                   (2, 12, 16, 16, 3), (1, 48, 8, 8, 3), (1, 3, 5, 5, 7),
+                                   # many channels (register-tiled kernel): ragged widths, several bands per image,
+                                   # several images per CTA, channel counts off the tile sizes, every k it serves
+                                   (3, 5, 7, 9, 2), (2, 13, 20, 20, 4), (1, 33, 6, 10, 5), (1, 6, 40, 36, 3), (2, 7, 5, 5, 1),
+                                   (5, 96, 8, 8, 5), (1, 8, 3, 250, 3), (1, 8, 3, 260, 3), (9, 17, 4, 4, 3), (2, 6, 9, 9, 7)],
+                         ids=lambda s: "x".join(map(str, s)))
 def test_masked_conv_matches_oracle(B, oracle, shape, path):
     """y = f(x) on its own (the sampling direction), junk in the masked-out kernel entries."""
     import torch
