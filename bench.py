@@ -395,6 +395,31 @@ def run_table(args):
         print(json.dumps(r))
 
 
+def run_sweep(args):
+    """The paper's ablation axes at three channels (kernel size, image side, batch size): microseconds per call,
+    and per diagonal, against the O(m k^2) model of Table 1 (human-readable, one JSON object per shape)."""
+    import torch
+    from paper_2410_14634_b200 import binding, workloads
+    device = torch.device("cuda:0")
+    cases = [("k", 32, 3, 32, k) for k in (2, 3, 5, 7, 9, 11)]
+    cases += [("side", 32, 3, m, 3) for m in (16, 32, 64, 128, 256)]
+    cases += [("batch", b, 3, 32, 3) for b in (1, 4, 16, 64, 128, 256)]
+    for axis, Bn, C, m, k in cases:
+        w, y, gx = workloads.make_custom(900 + Bn + m + k, Bn, C, m, m, k, sigma=0.02)
+        shape = workloads.Shape(f"sweep_{axis}_B{Bn}_m{m}_k{k}", 0, Bn, C, m, m, k, 0.02, 0.8, 1.2, 0)
+        ds = DeviceStep(shape, w, y, gx, device)
+        path = binding.invconv_path_for(Bn, C, m, m, k)
+        steps = max(3, min(args.steps, 200 if path != binding.PATH_GENERIC else 10))
+        ms_f, _ = ds.time_graphs("fwd", steps, min(args.warmup, 5))
+        ms_b, _ = ds.time_graphs("bwd", steps, min(args.warmup, 5))
+        tf, tb = ms_f / steps * 1e3, ms_b / steps * 1e3
+        print(json.dumps({"axis": axis, "B": Bn, "C": C, "side": m, "k": k, "path": path, "t_fwd_us": round(tf, 2),
+                          "t_bwd_us": round(tb, 2), "fwd_ns_per_diagonal": round(tf * 1e3 / (2 * m - 1), 1),
+                          "images_per_s": round(Bn / ((tf + tb) * 1e-6))}), flush=True)
+        del ds
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -403,6 +428,7 @@ def main():
     ap.add_argument("--workload", default="mnist")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--table", action="store_true", help="time every benchmark shape on one GPU")
+    ap.add_argument("--sweep", action="store_true", help="time the ablation axes (kernel size, image side, batch) at C=3")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -411,6 +437,9 @@ def main():
         return
     if args.table:
         run_table(args)
+        return
+    if args.sweep:
+        run_sweep(args)
         return
     run_ours(args, rank, world)
 

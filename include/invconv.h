@@ -94,6 +94,27 @@ int masked_conv_forward(const float* x, const float* w, float* y,
  * negative.  logdet points to ONE device float. */
 int invconv_logdet(const float* w, float* logdet, int C, int H, int W, int k, void* stream);
 
+/* The two calls of a flow layer's training step with the log-det folded in
+ * (Section 4: the layer contributes its log-det to the likelihood):
+ *
+ * invconv_forward_logdet = invconv_forward followed, on the same stream, by
+ *   invconv_logdet into logdet[0] (ONE device float; the log-det of f -- the
+ *   layer z = f^{-1}(y) contributes its negative).
+ *
+ * invconv_backward_logdet = invconv_backward followed by
+ *   grad_w[c][c][k-1][k-1] += grad_logdet[0] * H*W / w[c][c][k-1][k-1]  for every c,
+ *   the derivative of grad_logdet[0] * logdet with respect to w (zero for every
+ *   other entry).  grad_logdet points to ONE device float (the upstream
+ *   gradient of the loss with respect to the log-det value returned above);
+ *   grad_w must be non-NULL here.
+ * Argument rules, scratch and errors are those of invconv_forward/backward;
+ * the extra work is one single-warp kernel launch per call. */
+int invconv_forward_logdet(const float* y, const float* w, float* x, float* logdet,
+                           int B, int C, int H, int W, int k, void* stream);
+int invconv_backward_logdet(const float* grad_x, const float* x, const float* w, const float* grad_logdet,
+                            float* grad_y, float* grad_w,
+                            int B, int C, int H, int W, int k, void* stream);
+
 /* Scratch bytes a forward or backward call of this shape needs (0 if none).
  * Same value for both directions. */
 size_t invconv_workspace_bytes(int B, int C, int H, int W, int k);

@@ -44,6 +44,8 @@ def _load():
             fn.restype = None
         lib.oracle_logdet.argtypes = [dp, ci, ci, ci, ci]
         lib.oracle_logdet.restype = ctypes.c_double
+        lib.oracle_logdet_grad_w.argtypes = [dp, dp, ci, ci, ci, ci]
+        lib.oracle_logdet_grad_w.restype = None
         _lib = lib
     return _lib
 
@@ -116,3 +118,13 @@ def logdet(w, H: int, W: int) -> float:
     if w.ndim != 4:
         raise ValueError("kernel is [C,C,k,k]")
     return float(_load().oracle_logdet(_ptr(w), w.shape[0], H, W, w.shape[2]))
+
+
+def logdet_grad_w(w, H: int, W: int) -> np.ndarray:
+    """d logdet / d w: H*W / w[c,c,k-1,k-1] on the channel diagonal of the bottom-right tap, 0 elsewhere."""
+    w = _f64(w)
+    if w.ndim != 4:
+        raise ValueError("kernel is [C,C,k,k]")
+    gw = np.empty_like(w)
+    _load().oracle_logdet_grad_w(_ptr(w), _ptr(gw), w.shape[0], H, W, w.shape[2])
+    return gw

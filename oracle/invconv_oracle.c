@@ -163,3 +163,14 @@ double oracle_logdet(const double *w, int C, int H, int W, int k)
         s += log(fabs(w[WIDX(c, c, k - 1, k - 1, C, k)]));
     return (double)H * (double)W * s;
 }
+
+/* d logdet / d w, same shape as w: H*W / w[c][c][k-1][k-1] on the channel
+ * diagonal of the bottom-right tap, 0 everywhere else (derivative of
+ * H*W*sum_c log|w_cc|; the flow's loss adds a multiple of the log-det to the
+ * likelihood, Section 4). */
+void oracle_logdet_grad_w(const double *w, double *gw, int C, int H, int W, int k)
+{
+    for (int i = 0; i < C * C * k * k; ++i) gw[i] = 0.0;
+    for (int c = 0; c < C; ++c)
+        gw[WIDX(c, c, k - 1, k - 1, C, k)] = (double)H * (double)W / w[WIDX(c, c, k - 1, k - 1, C, k)];
+}

@@ -44,6 +44,8 @@ def lib() -> ctypes.CDLL:
         L.invconv_backward.argtypes = [fp, fp, fp, fp, fp, ci, ci, ci, ci, ci, vp]
         L.masked_conv_forward.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, vp]
         L.invconv_logdet.argtypes = [fp, fp, ci, ci, ci, ci, vp]
+        L.invconv_forward_logdet.argtypes = [fp, fp, fp, fp, ci, ci, ci, ci, ci, vp]
+        L.invconv_backward_logdet.argtypes = [fp, fp, fp, fp, fp, fp, ci, ci, ci, ci, ci, vp]
         L.invconv_workspace_bytes.argtypes = [ci] * 5
         L.invconv_workspace_bytes.restype = sz
         L.invconv_forward_ws.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, vp, sz, vp]
@@ -63,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.invconv_kernel_launch_count.argtypes = []
         L.invconv_kernel_launch_count.restype = ctypes.c_ulonglong
         for name in ("invconv_forward", "invconv_backward", "masked_conv_forward", "invconv_logdet",
+                     "invconv_forward_logdet", "invconv_backward_logdet",
                      "invconv_forward_ws", "invconv_backward_ws", "invconv_step_host", "invconv_set_path",
                      "invconv_path_for", "invconv_get_status", "invconv_probe_step_latency", "invconv_version"):
             getattr(L, name).restype = ci
@@ -192,6 +195,39 @@ def invconv_logdet(w: torch.Tensor, H: int, W: int, out: Optional[torch.Tensor] 
         _check(lib().invconv_logdet(w.data_ptr(), ld.data_ptr(), int(w.shape[0]), H, W, k,
                                     _stream_ptr(stream, w.device)), "invconv_logdet")
     return ld
+
+
+def invconv_forward_logdet(y: torch.Tensor, w: torch.Tensor, stream: Optional[torch.cuda.Stream] = None):
+    """(x, logdet): x = f^{-1}(y) and the log-det of f in one call."""
+    _act(y, "y")
+    B, C, H, W = y.shape
+    k = _kern(w, C)
+    x = torch.empty_like(y)
+    ld = torch.empty(1, dtype=torch.float32, device=y.device)
+    with torch.cuda.device(y.device):
+        _check(lib().invconv_forward_logdet(y.data_ptr(), w.data_ptr(), x.data_ptr(), ld.data_ptr(), B, C, H, W, k,
+                                            _stream_ptr(stream, y.device)), "invconv_forward_logdet")
+    return x, ld
+
+
+def invconv_backward_logdet(grad_x: torch.Tensor, x: torch.Tensor, w: torch.Tensor, grad_logdet: torch.Tensor,
+                            stream: Optional[torch.cuda.Stream] = None):
+    """(grad_y, grad_w) with grad_logdet * d logdet / d w added to grad_w; grad_logdet is a one-element fp32
+    CUDA tensor (the upstream gradient with respect to the log-det)."""
+    _act(grad_x, "grad_x")
+    _act(x, "x")
+    if grad_x.shape != x.shape:
+        raise ValueError("grad_x and x must have the same shape")
+    if grad_logdet.dtype != torch.float32 or grad_logdet.numel() != 1 or not grad_logdet.is_cuda:
+        raise ValueError("grad_logdet must be a one-element fp32 CUDA tensor")
+    B, C, H, W = x.shape
+    k = _kern(w, C)
+    gy, gw = torch.empty_like(grad_x), torch.empty_like(w)
+    with torch.cuda.device(x.device):
+        _check(lib().invconv_backward_logdet(grad_x.data_ptr(), x.data_ptr(), w.data_ptr(), grad_logdet.data_ptr(),
+                                             gy.data_ptr(), gw.data_ptr(), B, C, H, W, k,
+                                             _stream_ptr(stream, x.device)), "invconv_backward_logdet")
+    return gy, gw
 
 
 class HostStep:

@@ -165,4 +165,15 @@ __global__ void logdet_kernel(const float* __restrict__ wgt, float* __restrict__
     if (threadIdx.x == 0) out[0] = (float)((double)H * (double)W * s);
 }
 
+// grad_w[c][c][k-1][k-1] += grad_logdet * H*W / w[c][c][k-1][k-1]: the derivative of grad_logdet * logdet.
+__global__ void logdet_grad_kernel(const float* __restrict__ wgt, const float* __restrict__ grad_logdet,
+                                   float* __restrict__ grad_w, int C, int H, int W, int k)
+{
+    const float g = grad_logdet[0] * (float)H * (float)W;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) {
+        const int i = w_index(c, c, k - 1, k - 1, C, k);
+        grad_w[i] += g / wgt[i];
+    }
+}
+
 }  // namespace invconv

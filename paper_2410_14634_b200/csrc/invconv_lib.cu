@@ -650,6 +650,25 @@ int invconv_logdet(const float* w, float* logdet, int C, int H, int W, int k, vo
     return check_launch();
 }
 
+int invconv_forward_logdet(const float* y, const float* w, float* x, float* logdet,
+                           int B, int C, int H, int W, int k, void* stream)
+{
+    if (!logdet) return INVCONV_BAD_ARG;
+    const int rc = invconv_forward(y, w, x, B, C, H, W, k, stream);
+    if (rc) return rc;
+    return invconv_logdet(w, logdet, C, H, W, k, stream);
+}
+
+int invconv_backward_logdet(const float* grad_x, const float* x, const float* w, const float* grad_logdet,
+                            float* grad_y, float* grad_w, int B, int C, int H, int W, int k, void* stream)
+{
+    if (!grad_logdet || !grad_w) return INVCONV_BAD_ARG;
+    const int rc = invconv_backward(grad_x, x, w, grad_y, grad_w, B, C, H, W, k, stream);
+    if (rc) return rc;
+    logdet_grad_kernel<<<1, 128, 0, as_stream(stream)>>>(w, grad_logdet, grad_w, C, H, W, k);
+    return check_launch();
+}
+
 size_t invconv_step_scratch_bytes(int B, int C, int H, int W, int k)
 {
     if (check_shape(B, C, H, W, k) != INVCONV_OK) return 0;

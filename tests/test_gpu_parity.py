@@ -196,6 +196,33 @@ def test_masked_conv_matches_oracle(B, oracle, shape, path):
     assert nmax_err(y.cpu().numpy(), oracle.masked_conv(x, w)) <= 1e-5
 
 
+@pytest.mark.parametrize("shape", [(4, 3, 16, 16, 3), (3, 1, 28, 28, 3), (2, 12, 8, 8, 3), (2, 5, 6, 7, 2)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_training_step_calls_with_the_log_det_folded_in(B, oracle, shape):
+    """invconv_forward_logdet / invconv_backward_logdet against the oracle's x, logdet, grad_y and
+    grad_w + grad_logdet * d logdet / d w."""
+    import torch
+    Bn, C, H, W, k = shape
+    w, y, gx = workloads.make_custom(500 + sum(shape), Bn, C, H, W, k, sigma=0.05 / np.sqrt(C))
+    gl = -0.37
+    x, ld = B.invconv_forward_logdet(dev(y), dev(w))
+    gy, gw = B.invconv_backward_logdet(dev(gx), x, dev(w), torch.tensor([gl], dtype=torch.float32, device="cuda"))
+    torch.cuda.synchronize()
+    assert B.invconv_get_status() == 0
+    x_ref = oracle.invconv_forward(y, w)
+    gy_ref, gw_ref = oracle.invconv_backward(gx, x_ref, w)
+    gw_ref = gw_ref + gl * oracle.logdet_grad_w(w, H, W)
+    ld_ref = oracle.logdet(w, H, W)
+    assert nmax_err(x.cpu().numpy(), x_ref) <= TOL_X
+    assert nmax_err(gy.cpu().numpy(), gy_ref) <= TOL_X
+    assert nmax_err(gw.cpu().numpy(), gw_ref) <= TOL_GW
+    assert abs(float(ld.item()) - ld_ref) <= 1e-5 * max(abs(ld_ref), H * W * 1e-3)
+    # the diagonal term alone, where it dominates: compare the difference to plain backward
+    _, gw0 = B.invconv_backward(dev(gx), x, dev(w))
+    d = (gw - gw0).cpu().numpy().astype(np.float64)
+    assert nmax_err(d, gl * oracle.logdet_grad_w(w, H, W)) <= 1e-5
+
+
 def test_empty_batch_is_a_no_op_and_zeroes_grad_w(B):
     import torch
     w = dev(workloads.make_custom(9, 1, 2, 4, 4, 3)[0])

@@ -346,3 +346,23 @@ def test_logdet_scaling_law():
     w2 = w.copy()
     w2[np.arange(C), np.arange(C), k - 1, k - 1] *= s
     assert abs(api.logdet(w2, H, W) - api.logdet(w, H, W) - H * W * C * np.log(s)) < 1e-12 * H * W * C
+
+
+@pytest.mark.parametrize("B,C,H,W,k", TINY)
+def test_logdet_gradient_matches_slogdet_differences(B, C, H, W, k):
+    """d logdet / d w against central differences of numpy's slogdet of the dense matrix, entry by entry
+    (entries outside the mask and off the bottom-right tap's diagonal do not enter M's diagonal: 0)."""
+    w, _, _ = tiny_inputs(18, B, C, H, W, k)
+    w[C - 1, C - 1, k - 1, k - 1] *= -1.0
+    g = api.logdet_grad_w(w, H, W)
+    eps = 1e-6
+    for idx in np.ndindex(*w.shape):
+        co, ci, a, b = idx
+        if a == k - 1 and b == k - 1 and ci > co:
+            assert g[idx] == 0.0                   # masked out: not part of M
+            continue
+        wp, wm = w.copy(), w.copy()
+        wp[idx] += eps
+        wm[idx] -= eps
+        fd = (np.linalg.slogdet(dense.dense_matrix(wp, H, W))[1] - np.linalg.slogdet(dense.dense_matrix(wm, H, W))[1]) / (2 * eps)
+        assert abs(g[idx] - fd) < 1e-6 * max(1.0, abs(fd)), (idx, g[idx], fd)
