@@ -136,7 +136,14 @@ __global__ void __launch_bounds__(256) gradw_reduce_kernel(const float* __restri
     const int NA = K * K * C * C;
     for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < NA; e += gridDim.x * blockDim.x) {
         float s = 0.f;
-        for (int b = 0; b < nbc; ++b) s += __ldcg(partials + (size_t)b * NA + e);
+        for (int b0 = 0; b0 < nbc; b0 += 8) {              // eight loads in flight; the sum stays in share order
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = __ldcg(partials + (size_t)min(b0 + q, nbc - 1) * NA + e);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (b0 + q < nbc) s += v[q];
+        }
         const int ci = e % C, co = (e / C) % C, tap = e / (C * C);
         const int dh = tap / K, dw = tap % K;
         grad_w[((co * C + ci) * K + (K - 1 - dh)) * K + (K - 1 - dw)] = (tap == 0 && ci > co) ? 0.f : -s;
