@@ -58,8 +58,9 @@ constexpr size_t kMaxDynSmem = 226 * 1024;   // 227 KiB per CTA minus the kernel
 struct WarpPlan {
     bool ok = false;
     bool glb = false;      // image too large for shared memory: operands stay in global memory
+    bool ring = false;     // ... and a ring of 128 columns per warp fits: streamed through shared memory
     int nb = 0, ipc = 0, grid = 0;
-    size_t smem = 0;
+    size_t smem = 0, smem_ring = 0;
 };
 
 template <int C, int K>
@@ -79,6 +80,8 @@ WarpPlan plan_warp_ck(int B, int H, int W, bool bwd)
         pl.glb = true;
         pl.smem = warp_kernel_smem<C, K>(H, W, pl.nb, 1, bwd, true);
         if (pl.smem > kMaxDynSmem) return pl;
+        pl.smem_ring = warp_kernel_smem<C, K>(H, W, pl.nb, 1, bwd, true, true);
+        pl.ring = pl.smem_ring <= kMaxDynSmem;
     }
     pl.ipc = ipc;
     pl.grid = (B + ipc - 1) / ipc;
@@ -108,16 +111,20 @@ int set_smem_limit(Kern kern, size_t smem)
 template <int C, int K, bool BWD>
 int launch_warp_ck(const WarpPlan& pl, WarpParams prm, cudaStream_t st)
 {
-    auto kern = pl.glb ? warp_wavefront_kernel<C, K, BWD, true, true>
-                       : (pl.nb > 1 ? warp_wavefront_kernel<C, K, BWD, true> : warp_wavefront_kernel<C, K, BWD, false>);
-    const int rc = set_smem_limit(kern, pl.smem);
+    // global-memory mode: streamed through a shared-memory ring unless grad_w rides along in the wavefront
+    const bool ring = pl.glb && pl.ring && prm.grad_w == nullptr && std::getenv("INVCONV_NO_RING") == nullptr;
+    auto kern = ring ? warp_wavefront_kernel<C, K, BWD, true, true, true>
+                     : (pl.glb ? warp_wavefront_kernel<C, K, BWD, true, true>
+                               : (pl.nb > 1 ? warp_wavefront_kernel<C, K, BWD, true> : warp_wavefront_kernel<C, K, BWD, false>));
+    const size_t smem = ring ? pl.smem_ring : pl.smem;
+    const int rc = set_smem_limit(kern, smem);
     if (rc) return rc;
     // Programmatic dependent launch: the kernel may be scheduled while its predecessor on the stream drains;
     // it touches no global memory before griddepcontrol.wait, which waits for that predecessor to complete.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(pl.grid);
     cfg.blockDim = dim3(pl.nb * pl.ipc * 32);
-    cfg.dynamicSmemBytes = pl.smem;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -220,6 +227,7 @@ int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const fl
                            reinterpret_cast<uintptr_t>(xsaved)) & 15) == 0;
     prm.bulk = (aligned && chw % 4 == 0) ? 1 : 0;
     prm.glb = pl.glb ? 1 : 0;
+    prm.vec = (aligned && g.W % 4 == 0) ? 1 : 0;
     int rc = INVCONV_UNSUPPORTED;
 #define X(CC, KK)                                                                         \
     if (g.C == CC && g.k == KK)                                                           \

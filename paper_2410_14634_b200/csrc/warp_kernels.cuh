@@ -34,6 +34,10 @@
 #include "common.cuh"
 #include "tma.cuh"
 
+#ifndef INVCONV_UNROLL_K5
+#define INVCONV_UNROLL_K5 4      // unroll factor (in units of K-1 steps) of the one-channel 5x5 step loop
+#endif
+
 namespace invconv {
 
 struct WarpParams {
@@ -49,6 +53,7 @@ struct WarpParams {
     int ipc;               // images per CTA
     int bulk;              // images are 16-byte aligned multiples of 16 bytes
     int glb;               // images stay in global memory (too large for shared memory)
+    int vec;               // image rows are 16-byte aligned multiples of 16 bytes (ring mode: 16-byte copies)
 };
 
 template <int C> struct ColVec;
@@ -157,13 +162,95 @@ __device__ void build_transformed_kernel(const float* __restrict__ w, float* As)
 // written to, global memory directly (each lane walks its own row, so a 32-byte sector is fetched once and
 // then hit in L1 for eight steps; sectors are prefetched two ahead), and the K-1 bottom rows of every row
 // block go to a small shared-memory buffer `bnd` ([block][channel][row][W]) for the block below.
-template <int C, int K, bool MULTI, bool GW, bool GLB = false>
+//
+// RING = true (with GLB and MULTI, never GW) streams such images through shared memory instead: every warp
+// owns a ring of 128 physical columns of its 32 rows (four tiles of 32 columns; per channel kRingCh floats,
+// row stride 128, slot = physical column & 127, so the skewed accesses of the lanes stay conflict-free).
+// Every 32 steps the warp (a) waits for the tile it asked for 32 steps earlier, (b) writes the tile that all
+// of its lanes have finished (two tiles back) to global memory with coalesced stores, and (c) asks for the
+// tile two ahead with asynchronous copies into the slot just freed.  The step itself is the shared-memory
+// step: no global access on the dependent chain.  `vec` says whether rows are 16-byte aligned multiples of
+// 16 bytes (16-byte copies and stores), else single floats are moved.
+constexpr int kRingCh = 32 * 128 + 32;       // floats per channel of one warp's ring; the tail is a scratch slot
+
+// Tile t of the ring (logical columns 32t .. 32t+31 of the walk) as physical columns: first column and count.
+__device__ __forceinline__ void ring_tile_cols(int t, int W, int sgn, int& base, int& lo, int& hi)
+{
+    base = sgn > 0 ? 32 * t : W - 32 * (t + 1);      // may be negative for the last tile of a reversed walk
+    lo = max(base, 0);
+    hi = min(base + 32, W);
+}
+
+template <int C>
+__device__ __forceinline__ void ring_load_tile(float* ring, const float* rin, int t, int H, int W, int sgn, int j,
+                                               int rows, int lane, bool vec)
+{
+    int base, lo, hi;
+    ring_tile_cols(t, W, sgn, base, lo, hi);
+    const int HW = H * W;
+    if (vec) {
+#pragma unroll
+        for (int c = 0; c < C; ++c)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int v = i * 32 + lane, row = v >> 3, col = base + 4 * (v & 7);
+                const int pr = sgn > 0 ? 32 * j + row : H - 1 - (32 * j + row);
+                const bool ok = row < rows && col >= lo && col < hi;
+                cp_async_f32x4(ring + c * kRingCh + row * 128 + (col & 127), rin + (ok ? c * HW + pr * W + col : 0), ok);
+            }
+    } else {
+        const int col = base + lane;
+        const bool okc = col >= lo && col < hi;
+#pragma unroll
+        for (int c = 0; c < C; ++c)
+#pragma unroll 8
+            for (int row = 0; row < 32; ++row) {
+                const int pr = sgn > 0 ? 32 * j + row : H - 1 - (32 * j + row);
+                const bool ok = okc && row < rows;
+                cp_async_f32(ring + c * kRingCh + row * 128 + (col & 127), rin + (ok ? c * HW + pr * W + col : 0), ok);
+            }
+    }
+}
+
+template <int C>
+__device__ __forceinline__ void ring_store_tile(const float* ring, float* out, int t, int H, int W, int sgn, int j,
+                                                int rows, int lane, bool vec)
+{
+    int base, lo, hi;
+    ring_tile_cols(t, W, sgn, base, lo, hi);
+    const int HW = H * W;
+    if (vec) {
+#pragma unroll
+        for (int c = 0; c < C; ++c)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int v = i * 32 + lane, row = v >> 3, col = base + 4 * (v & 7);
+                const int pr = sgn > 0 ? 32 * j + row : H - 1 - (32 * j + row);
+                const float4 val = *reinterpret_cast<const float4*>(ring + c * kRingCh + row * 128 + (col & 127));
+                if (row < rows && col >= lo && col < hi) *reinterpret_cast<float4*>(out + c * HW + pr * W + col) = val;
+            }
+    } else {
+        const int col = base + lane;
+        const bool okc = col >= lo && col < hi;
+#pragma unroll
+        for (int c = 0; c < C; ++c)
+#pragma unroll 8
+            for (int row = 0; row < 32; ++row) {
+                const int pr = sgn > 0 ? 32 * j + row : H - 1 - (32 * j + row);
+                const float val = ring[c * kRingCh + row * 128 + (col & 127)];
+                if (okc && row < rows) out[c * HW + pr * W + col] = val;
+            }
+    }
+}
+
+template <int C, int K, bool MULTI, bool GW, bool GLB = false, bool RING = false>
 __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int H, int W, int origin, int sgn,
                                                 int j, volatile int* progress, int lane,
                                                 const float* xs = nullptr, float* gw_dst = nullptr,
                                                 const float* rin = nullptr, float* bnd = nullptr, int nb = 1,
-                                                int dummy_idx = 0)
+                                                int dummy_idx = 0, float* ring = nullptr, bool vec = false)
 {
+    static_assert(!RING || (GLB && MULTI && !GW), "the ring serves the global-memory mode without fused grad_w");
     if (!GLB) rin = img;
     using S = WarpShape<C, K>;
     constexpr int KM = K - 1;
@@ -201,12 +288,38 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
 #pragma unroll
     for (int i = 0; i < (GW ? S::NA : 1); ++i) gacc[i] = 0.f;
     int p = origin + sgn * ((32 * j + lane) * W - lane);    // offset of (lh, lw) at step 0
+    int pcol = sgn > 0 ? -lane : W - 1 + lane;              // RING: physical column of (lh, lw) at step 0
+    const int rbase = lane * 128;
+    const int ntiles = (W + 31) >> 5;
+    int next_flush = 0;
+    if constexpr (RING) {
+        ring_load_tile<C>(ring, rin, 0, H, W, sgn, j, rows, lane, vec);
+        if (ntiles > 1) ring_load_tile<C>(ring, rin, 1, H, W, sgn, j, rows, lane, vec);
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncwarp();
+    }
     float rnext[C];
 #pragma unroll
-    for (int c = 0; c < C; ++c) rnext[c] = (lane == 0 && Wl > 0) ? rin[c * HW + p] : 0.f;
+    for (int c = 0; c < C; ++c) {
+        if constexpr (RING) rnext[c] = (lane == 0 && Wl > 0) ? ring[c * kRingCh + rbase + (pcol & 127)] : 0.f;
+        else rnext[c] = (lane == 0 && Wl > 0) ? rin[c * HW + p] : 0.f;
+    }
 
-#pragma unroll(C >= 3 ? 2 : 4)
+    constexpr int UNR = C >= 3 ? 2 : (K == 5 ? INVCONV_UNROLL_K5 : 4);
+#pragma unroll(UNR)
     for (int s0 = 0; s0 < nsteps_up; s0 += KM) {
+        if constexpr (RING) {
+            if ((s0 & 31) == 0) {
+                const int t = s0 >> 5;
+                cp_async_wait<0>();                      // tile t+1, asked for 32 steps ago
+                __syncwarp();
+                if (t >= 2 && t - 2 < ntiles) { ring_store_tile<C>(ring, img, t - 2, H, W, sgn, j, rows, lane, vec); next_flush = t - 1; }
+                __syncwarp();
+                if (t + 2 < ntiles) ring_load_tile<C>(ring, rin, t + 2, H, W, sgn, j, rows, lane, vec);
+                cp_async_commit();
+            }
+        }
         if constexpr (MULTI) {
             if (j > 0 && (s0 & 7) == 0) {
                 const int need = min(s0 + 39, prod_steps);
@@ -215,7 +328,10 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
                 while (progress[j - 1] < need) {
                     if (++spins > kMaxSpins) { ok = false; break; }
                 }
-                if (!__all_sync(0xffffffffu, ok)) return false;
+                if (!__all_sync(0xffffffffu, ok)) {
+                    if constexpr (RING) cp_async_wait<0>();
+                    return false;
+                }
                 __threadfence_block();
             }
         }
@@ -236,7 +352,11 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
             }
             {
                 const bool act1 = (ulw + 1u) < Wl;
-                if constexpr (GLB) {
+                if constexpr (RING) {
+                    const int rn = act1 ? rbase + ((pcol + sgn) & 127) : 32 * 128;   // inactive lanes: the scratch slot
+#pragma unroll
+                    for (int c = 0; c < C; ++c) { const float t = ring[c * kRingCh + rn]; rnext[c] = act1 ? t : 0.f; }
+                } else if constexpr (GLB) {
 #pragma unroll
                     for (int c = 0; c < C; ++c) rnext[c] = act1 ? rin[c * HW + p + sgn] : 0.f;
                 } else {
@@ -244,7 +364,7 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
 #pragma unroll
                     for (int c = 0; c < C; ++c) { const float t = rin[c * HW + pn]; rnext[c] = act1 ? t : 0.f; }
                 }
-                if constexpr (GLB) {
+                if constexpr (GLB && !RING) {
                     if (((ulw + 1u) & 7u) == 0u && (ulw + 17u) < Wl) {
 #pragma unroll
                         for (int c = 0; c < C; ++c) {
@@ -351,7 +471,17 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
 #pragma unroll
                 for (int a = 0; a < C; ++a) img[active ? a * HW + p : dummy_idx] = acc[a];
             }
-            if (GLB && active) {
+            if constexpr (RING) {
+                const int ro = active ? rbase + (pcol & 127) : 32 * 128;
+#pragma unroll
+                for (int a = 0; a < C; ++a) ring[a * kRingCh + ro] = acc[a];
+                // the K-1 bottom rows also go to the boundary buffer of the block below (its last float is scratch)
+                const bool pub = active && lane >= 32 - KM && j + 1 < nb;
+#pragma unroll
+                for (int a = 0; a < C; ++a)
+                    bnd[pub ? ((j * C + a) * KM + (lane - (32 - KM))) * W + (int)ulw : nb * C * KM * W] = acc[a];
+            }
+            if (GLB && !RING && active) {
 #pragma unroll
                 for (int a = 0; a < C; ++a) img[a * HW + p] = acc[a];
                 if constexpr (GLB && MULTI) {
@@ -385,6 +515,7 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
                 for (int d = 0; d < KM; ++d) up[d][b][u] = nu[d][b];
             }
             p += sgn;
+            pcol += sgn;
         }
         if constexpr (MULTI) {
             if (((s0 + KM) & 7) == 0) {
@@ -398,6 +529,11 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
         __threadfence_block();
         __syncwarp();
         if (lane == 0) progress[j] = prod_steps;
+    }
+    if constexpr (RING) {
+        cp_async_wait<0>();
+        __syncwarp();
+        for (int t = next_flush; t < ntiles; ++t) ring_store_tile<C>(ring, img, t, H, W, sgn, j, rows, lane, vec);
     }
     if constexpr (GW) {
         // rows above the image never existed for the first lanes of the first block: drop what they gathered
@@ -494,10 +630,10 @@ __device__ __forceinline__ void grad_w_block(const float* gy, const float* xs, i
 template <int C, int K>
 struct WarpSmem {
     using S = WarpShape<C, K>;
-    int as_off, bar_off, prog_off, red_off, img_off, imgf, bnd_off, dummy_off, total;
+    int as_off, bar_off, prog_off, red_off, img_off, imgf, bnd_off, dummy_off, ring_off, total;
     // Hg > 0: the images stay in global memory (H = 0 is passed) and only the boundary rows between the row
-    // blocks of one image live here.
-    __host__ __device__ WarpSmem(int H, int W, int nb, int ipc, bool bwd, int Hg = 0)
+    // blocks of one image live here; ring: every warp also owns a ring of 128 columns of its rows.
+    __host__ __device__ WarpSmem(int H, int W, int nb, int ipc, bool bwd, int Hg = 0, bool ring = false)
     {
         auto up32 = [](int v) { return (v + 31) & ~31; };
         as_off = 0;
@@ -507,12 +643,13 @@ struct WarpSmem {
         img_off = red_off + (bwd ? up32(nb * ipc * S::NA) : 0);
         imgf = up32(C * H * W);
         bnd_off = img_off + imgf * ipc * (bwd ? 2 : 1);
-        dummy_off = bnd_off + (Hg > 0 ? up32(nb * C * (K - 1) * W) : 0);
-        total = dummy_off + 32;
+        dummy_off = bnd_off + (Hg > 0 ? up32(nb * C * (K - 1) * W + 1) : 0);
+        ring_off = dummy_off + 32;
+        total = ring_off + (ring ? nb * ipc * C * kRingCh : 0);
     }
 };
 
-template <int C, int K, bool BWD, bool MULTI, bool GLB = false>
+template <int C, int K, bool BWD, bool MULTI, bool GLB = false, bool RING = false>
 __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
 {
     using S = WarpShape<C, K>;
@@ -523,7 +660,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     const int li = warp / p.nb, j = warp - li * p.nb;  // image within the CTA, row block within the image
     const int n = blockIdx.x * p.ipc + li;             // image index
     const bool has_img = n < p.B;
-    const WarpSmem<C, K> lay(GLB ? 0 : H, W, p.nb, p.ipc, BWD, GLB ? H : 0);
+    const WarpSmem<C, K> lay(GLB ? 0 : H, W, p.nb, p.ipc, BWD, GLB ? H : 0, RING);
 
     float* As = smem + lay.as_off;
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + lay.bar_off);
@@ -543,7 +680,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     }
 
     constexpr bool FUSE_GW = (S::NA <= 81);   // few enough partial sums to ride along in the wavefront's registers
-    const bool want_gw = BWD && p.grad_w != nullptr;
+    const bool want_gw = BWD && !RING && p.grad_w != nullptr;     // the ring mode never carries grad_w
     const bool leader = has_img && j == 0 && lane == 0;
     // everything above touched no global memory; from here on the predecessor kernel's results are needed
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -584,7 +721,11 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
         ok = __all_sync(0xffffffffu, ok);
         WARP_TT(2);
         if (ok) {
-            if (BWD && FUSE_GW && want_gw)
+            if constexpr (RING)
+                ok = wavefront_block<C, K, MULTI, false, GLB, true>(img, As, H, W, BWD ? HW - 1 : 0, BWD ? -1 : 1, j,
+                                                                    progress + li * p.nb, lane, nullptr, nullptr, rin, bnd, p.nb,
+                                                                    dummy_idx, smem + lay.ring_off + warp * C * kRingCh, p.vec != 0);
+            else if (BWD && FUSE_GW && want_gw)
                 ok = wavefront_block<C, K, MULTI, BWD && FUSE_GW, GLB>(img, As, H, W, HW - 1, -1, j, progress + li * p.nb,
                                                                        lane, xs, red + warp * S::NA, rin, bnd, p.nb, dummy_idx);
             else
@@ -682,9 +823,9 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
 
 // Dynamic shared memory the kernel needs for a launch shape.
 template <int C, int K>
-inline size_t warp_kernel_smem(int H, int W, int nb, int ipc, bool bwd, bool glb = false)
+inline size_t warp_kernel_smem(int H, int W, int nb, int ipc, bool bwd, bool glb = false, bool ring = false)
 {
-    if (glb) return sizeof(float) * (size_t)WarpSmem<C, K>(0, W, nb, ipc, bwd, H).total;
+    if (glb) return sizeof(float) * (size_t)WarpSmem<C, K>(0, W, nb, ipc, bwd, H, ring).total;
     return sizeof(float) * (size_t)WarpSmem<C, K>(H, W, nb, ipc, bwd).total;
 }
 

@@ -100,6 +100,7 @@ EDGE = [  # (B, C, H, W, k)
     (2, 12, 5, 7, 3), (1, 16, 9, 9, 3), (1, 33, 4, 6, 3), (1, 24, 8, 8, 5), (1, 1, 40, 70, 7),
     (1, 2, 16, 16, 11), (1, 1, 65, 66, 3), (1, 3, 100, 20, 3), (5, 1, 28, 28, 3),
     (1, 3, 100, 200, 3), (2, 1, 250, 260, 5), (1, 2, 70, 500, 2),       # larger than shared memory: global-memory mode
+    (1, 1, 250, 257, 3), (1, 2, 130, 301, 5), (1, 4, 96, 180, 2), (1, 3, 200, 160, 3),   # ... ragged widths (4-byte ring copies), ring too large
 ]
 
 
