@@ -59,8 +59,10 @@ struct WarpPlan {
     bool ok = false;
     bool glb = false;      // image too large for shared memory: operands stay in global memory
     bool ring = false;     // ... and a ring of 128 columns per warp fits: streamed through shared memory
+    bool cs = false;       // channel-split walk available (lane = (row, output channel)); its own geometry below
     int nb = 0, ipc = 0, grid = 0;
-    size_t smem = 0, smem_ring = 0;
+    int nb_cs = 0, ipc_cs = 0, grid_cs = 0;
+    size_t smem = 0, smem_ring = 0, smem_cs = 0;
 };
 
 template <int C, int K>
@@ -86,6 +88,21 @@ WarpPlan plan_warp_ck(int B, int H, int W, bool bwd)
     pl.ipc = ipc;
     pl.grid = (B + ipc - 1) / ipc;
     pl.ok = true;
+    // channel-split walk: where the transformed kernel does not fit one lane's registers (C >= 3, 5x5)
+    if (C >= 3 && K == 5 && !pl.glb) {
+        const int rpw = 32 / C;
+        const int nbc = (H + rpw - 1) / rpw;
+        if (nbc <= 8) {
+            int ic = 8 / nbc;
+            if (ic < 1) ic = 1;
+            if (ic > B) ic = B > 0 ? B : 1;
+            while (ic > 1 && warp_kernel_smem<C, K>(H, W, nbc, ic, bwd) > kMaxDynSmem) --ic;
+            const size_t sm = warp_kernel_smem<C, K>(H, W, nbc, ic, bwd);
+            if (sm <= kMaxDynSmem) {
+                pl.cs = true; pl.nb_cs = nbc; pl.ipc_cs = ic; pl.grid_cs = (B + ic - 1) / ic; pl.smem_cs = sm;
+            }
+        }
+    }
     return pl;
 }
 
@@ -113,17 +130,29 @@ int launch_warp_ck(const WarpPlan& pl, WarpParams prm, cudaStream_t st)
 {
     // global-memory mode: streamed through a shared-memory ring unless grad_w rides along in the wavefront
     const bool ring = pl.glb && pl.ring && prm.grad_w == nullptr && std::getenv("INVCONV_NO_RING") == nullptr;
+    // channel-split walk (its own row-block geometry) unless grad_w rides along in the wavefront
+    bool cs = false;
+    if constexpr (C >= 3 && K == 5) cs = pl.cs && prm.grad_w == nullptr && std::getenv("INVCONV_NO_CS") == nullptr;
     auto kern = ring ? warp_wavefront_kernel<C, K, BWD, true, true, true>
                      : (pl.glb ? warp_wavefront_kernel<C, K, BWD, true, true>
                                : (pl.nb > 1 ? warp_wavefront_kernel<C, K, BWD, true> : warp_wavefront_kernel<C, K, BWD, false>));
-    const size_t smem = ring ? pl.smem_ring : pl.smem;
+    size_t smem = ring ? pl.smem_ring : pl.smem;
+    int nb = pl.nb, ipc = pl.ipc, grid = pl.grid;
+    if constexpr (C >= 3 && K == 5) {
+        if (cs) {
+            kern = pl.nb_cs > 1 ? warp_wavefront_kernel<C, K, BWD, true, false, false, true>
+                                : warp_wavefront_kernel<C, K, BWD, false, false, false, true>;
+            smem = pl.smem_cs; nb = pl.nb_cs; ipc = pl.ipc_cs; grid = pl.grid_cs;
+            prm.nb = nb; prm.ipc = ipc;
+        }
+    }
     const int rc = set_smem_limit(kern, smem);
     if (rc) return rc;
     // Programmatic dependent launch: the kernel may be scheduled while its predecessor on the stream drains;
     // it touches no global memory before griddepcontrol.wait, which waits for that predecessor to complete.
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(pl.grid);
-    cfg.blockDim = dim3(pl.nb * pl.ipc * 32);
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(nb * ipc * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

@@ -555,6 +555,166 @@ __device__ __forceinline__ bool wavefront_block(float* img, const float* As, int
     return true;
 }
 
+// Channel-split wavefront for kernels whose transformed taps do not fit one lane's registers (C >= 3 with
+// K = 5): lane = (row r, output channel a), 32 / C rows per warp.  A lane keeps only column a of every
+// (tap, input channel) -- K*K*C registers -- and computes one output channel of its row's pixel per step
+// (K*K*C FMAs instead of K*K*C*C).  The solved neighbours of ALL input channels are still needed: the C lanes
+// of a row exchange their new values by shuffles (so every lane of the row holds the row's C newest values),
+// and the rows above come by shuffles over C*(d+1) lanes.  Row blocks are RPW rows high, so an image needs
+// more warps and the skew between consecutive blocks is RPW steps instead of 32.
+// Images resident in shared memory only; grad_w never rides along here.
+template <int C, int K, bool MULTI>
+__device__ __forceinline__ bool wavefront_block_cs(float* img, const float* As, int H, int W, int origin, int sgn,
+                                                   int j, volatile int* progress, int lane, int dummy_idx)
+{
+    using S = WarpShape<C, K>;
+    constexpr int KM = K - 1, RPW = 32 / C;
+    constexpr int PUB = KM >= 4 ? KM : 4;                   // steps between progress checks / publications
+    const int HW = H * W;
+    const int r = lane / C, a = lane - r * C;
+    const int row0 = RPW * j;
+    const int rows = min(RPW, H - row0);
+    const int nsteps = W + rows - 1;
+    const int nsteps_up = (nsteps + PUB - 1) / PUB * PUB;
+    const int prod_steps = (W + RPW - 1 + PUB - 1) / PUB * PUB;
+    const unsigned Wl = r < rows ? (unsigned)W : 0u;        // active  <=>  (unsigned)lw < Wl
+    const bool first_block = !MULTI || j == 0;
+
+    float Ar[S::KK * C];                                    // column a of (tap, input channel b)
+#pragma unroll
+    for (int t = 0; t < S::KK * C; ++t) {
+        float col[C];
+        load_col<C>(As, t, col);
+        float v = col[0];
+#pragma unroll
+        for (int q = 1; q < C; ++q) v = a == q ? col[q] : v;
+        const int dh = t / (C * K);
+        const bool dead = first_block && dh >= 1 && r < dh;  // the row dh above lies outside the image
+        Ar[t] = dead ? 0.f : v;
+    }
+    float own[C][KM];          // slot (s mod KM) <- x[b][lh][lw] of step s, all input channels b
+    float up[KM][C][KM];       // slot (s mod KM) <- x[b][lh-1-d][lw] of step s
+#pragma unroll
+    for (int b = 0; b < C; ++b)
+#pragma unroll
+        for (int q = 0; q < KM; ++q) {
+            own[b][q] = 0.f;
+#pragma unroll
+            for (int d = 0; d < KM; ++d) up[d][b][q] = 0.f;
+        }
+    int p = origin + sgn * ((row0 + r) * W - r);            // offset of (lh, lw) at step 0
+    float rnext[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) rnext[c] = (r == 0 && Wl > 0) ? img[c * HW + p] : 0.f;
+
+#pragma unroll 1
+    for (int s0 = 0; s0 < nsteps_up; s0 += KM) {
+        if constexpr (MULTI) {
+            if (j > 0 && (s0 % PUB) == 0) {
+                const int need = min(s0 + PUB - 1 + RPW, prod_steps);
+                unsigned spins = 0;
+                bool ok = true;
+                while (progress[j - 1] < need) {
+                    if (++spins > kMaxSpins) { ok = false; break; }
+                }
+                if (!__all_sync(0xffffffffu, ok)) return false;
+                __threadfence_block();
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < KM; ++u) {
+            const unsigned ulw = (unsigned)(s0 + u - r);
+            const bool active = ulw < Wl;
+            float rr[C];
+#pragma unroll
+            for (int c = 0; c < C; ++c) rr[c] = rnext[c];
+            {
+                const bool act1 = (ulw + 1u) < Wl;
+                const int pn = act1 ? p + sgn : origin;      // inactive lanes read a valid dummy location: no branch
+#pragma unroll
+                for (int c = 0; c < C; ++c) { const float t = img[c * HW + pn]; rnext[c] = act1 ? t : 0.f; }
+            }
+            // newest column of the rows above.  Row lh-1 (on the dependent chain): by shuffle inside the block,
+            // from shared memory across blocks.  Rows lh-2 and further were solved at least two steps ago and are
+            // read back from the image in shared memory (this warp's own stores of earlier steps, or the block
+            // above, which the progress counter covers); lanes outside the image or not yet started get zeros.
+            float nu[KM][C];
+            __syncwarp();
+#pragma unroll
+            for (int b = 0; b < C; ++b) {
+                float v = __shfl_up_sync(0xffffffffu, own[b][(u - 1 + 2 * KM) % KM], C);
+                if constexpr (MULTI) {
+                    const bool edge = r == 0;
+                    const bool take = edge && j > 0 && active;
+                    const float vb = img[take ? b * HW + p - sgn * W : dummy_idx];
+                    v = edge ? (take ? vb : 0.f) : v;
+                }
+                nu[0][b] = v;
+            }
+#pragma unroll
+            for (int d = 1; d < KM; ++d) {
+                const bool have = active && (row0 + r - d - 1 >= 0);
+#pragma unroll
+                for (int b = 0; b < C; ++b) {
+                    const float t = img[have ? b * HW + p - sgn * (d + 1) * W : dummy_idx];
+                    nu[d][b] = have ? t : 0.f;
+                }
+            }
+            // everything off the dependent chain, on six independent accumulators (a lone accumulator would make
+            // every FMA wait four cycles for the one before it)
+            float pa[4] = {0.f, 0.f, 0.f, 0.f}, pn = 0.f, py = 0.f;
+#pragma unroll
+            for (int b = 0; b < C; ++b) py = fmaf(Ar[b], rr[b], py);
+            {
+                int q = 0;
+#pragma unroll
+                for (int dh = 0; dh < K; ++dh)
+#pragma unroll
+                    for (int dw = (dh == 0 ? 2 : 1); dw < K; ++dw)
+#pragma unroll
+                        for (int b = 0; b < C; ++b) {
+                            const int slot = (u - dw + 2 * KM) % KM;      // produced at step s - dw
+                            const float v = dh == 0 ? own[b][slot] : up[dh - 1][b][slot];
+                            pa[q & 3] = fmaf(-Ar[(dh * K + dw) * C + b], v, pa[q & 3]);
+                            ++q;
+                        }
+            }
+#pragma unroll
+            for (int d = KM - 1; d >= 1; --d)
+#pragma unroll
+                for (int b = 0; b < C; ++b) pn = fmaf(-Ar[((d + 1) * K) * C + b], nu[d][b], pn);
+            float acc = ((pa[0] + pa[1]) + (pa[2] + pa[3])) + (pn + py);
+            // the two taps on the true critical path: left neighbour, then the row above
+#pragma unroll
+            for (int b = 0; b < C; ++b) acc = fmaf(-Ar[1 * C + b], own[b][(u - 1 + 2 * KM) % KM], acc);
+#pragma unroll
+            for (int b = 0; b < C; ++b) acc = fmaf(-Ar[K * C + b], nu[0][b], acc);
+            img[active ? a * HW + p : dummy_idx] = acc;
+            // every lane of the row gets the row's C new values
+#pragma unroll
+            for (int b = 0; b < C; ++b) {
+                own[b][u] = __shfl_sync(0xffffffffu, acc, (r * C + b) & 31);
+#pragma unroll
+                for (int d = 0; d < KM; ++d) up[d][b][u] = nu[d][b];
+            }
+            p += sgn;
+        }
+        if constexpr (MULTI) {
+            if (((s0 + KM) % PUB) == 0) {
+                __threadfence_block();
+                __syncwarp();
+                if (lane == 0) progress[j] = s0 + KM;
+            }
+        }
+    }
+    if constexpr (MULTI) {
+        __threadfence_block();
+        __syncwarp();
+        if (lane == 0) progress[j] = prod_steps;
+    }
+    return true;
+}
+
 // grad_w partial of one row block, lane = column (Theorem 2 in closed form):
 //   part[((dh*K+dw)*C + co)*C + ci] = sum_{h in block, w} gy[co][h][w] * x[ci][h-dh][w-dw]
 // written to `dst` (shared memory, NA floats) by the lanes that end up owning each entry.
@@ -649,9 +809,10 @@ struct WarpSmem {
     }
 };
 
-template <int C, int K, bool BWD, bool MULTI, bool GLB = false, bool RING = false>
+template <int C, int K, bool BWD, bool MULTI, bool GLB = false, bool RING = false, bool CS = false>
 __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
 {
+    static_assert(!CS || (!GLB && !RING), "the channel-split walk serves images resident in shared memory");
     using S = WarpShape<C, K>;
     extern __shared__ __align__(128) float smem[];
     const int H = p.H, W = p.W, HW = H * W, CHW = C * HW;
@@ -680,7 +841,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     }
 
     constexpr bool FUSE_GW = (S::NA <= 81);   // few enough partial sums to ride along in the wavefront's registers
-    const bool want_gw = BWD && !RING && p.grad_w != nullptr;     // the ring mode never carries grad_w
+    const bool want_gw = BWD && !RING && !CS && p.grad_w != nullptr;     // ring and channel-split modes never carry grad_w
     const bool leader = has_img && j == 0 && lane == 0;
     // everything above touched no global memory; from here on the predecessor kernel's results are needed
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -721,7 +882,10 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
         ok = __all_sync(0xffffffffu, ok);
         WARP_TT(2);
         if (ok) {
-            if constexpr (RING)
+            if constexpr (CS)
+                ok = wavefront_block_cs<C, K, MULTI>(img, As, H, W, BWD ? HW - 1 : 0, BWD ? -1 : 1, j, progress + li * p.nb,
+                                                     lane, dummy_idx);
+            else if constexpr (RING)
                 ok = wavefront_block<C, K, MULTI, false, GLB, true>(img, As, H, W, BWD ? HW - 1 : 0, BWD ? -1 : 1, j,
                                                                     progress + li * p.nb, lane, nullptr, nullptr, rin, bnd, p.nb,
                                                                     dummy_idx, smem + lay.ring_off + warp * C * kRingCh, p.vec != 0);
