@@ -136,9 +136,13 @@ int invconv_backward_ws(const float* grad_x, const float* x, const float* w,
 
 /* One whole layer step from HOST buffers: copies y, w, grad_x to the device,
  * runs invconv_forward, invconv_backward and invconv_logdet there, and copies
- * x, grad_y, grad_w and the log-det back -- all enqueued on `stream`, no
+ * x, grad_y, grad_w and the log-det back -- enqueued on `stream`, no
  * synchronisation (use pinned host memory for truly asynchronous copies and
- * synchronise the stream before reading the outputs).
+ * synchronise the stream before reading the outputs).  The copy of grad_x in
+ * and of x out run on a library-owned side stream (one per device, created on
+ * first use) so that the two copy directions overlap each other and the
+ * kernels; the side stream is forked from and joined back into `stream` with
+ * events inside the call, so `stream` alone orders the whole step.
  *   *_host: host pointers (y, grad_x, x, grad_y: B*C*H*W floats; w, grad_w:
  *   C*C*k*k floats; logdet: 1 float).
  *   device_scratch: caller-owned device memory of at least

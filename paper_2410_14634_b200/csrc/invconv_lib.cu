@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 #include "invconv.h"
 
@@ -591,6 +592,31 @@ struct StreamScratch {
     ~StreamScratch() { if (p) cudaFreeAsync(p, st); }
 };
 
+// Side stream and events of invconv_step_host, one set per device, created on first use and kept.
+struct StepSide {
+    cudaStream_t side = nullptr;
+    cudaEvent_t start = nullptr, gx_in = nullptr, x_ready = nullptr, x_out = nullptr;
+    bool ok = false;
+};
+
+StepSide* step_side()
+{
+    static std::mutex mu;
+    static StepSide sides[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return nullptr; }
+    std::lock_guard<std::mutex> lock(mu);
+    StepSide& s = sides[dev];
+    if (!s.ok) {
+        bool good = cudaStreamCreateWithFlags(&s.side, cudaStreamNonBlocking) == cudaSuccess;
+        cudaEvent_t* evs[4] = {&s.start, &s.gx_in, &s.x_ready, &s.x_out};
+        for (cudaEvent_t* e : evs) good = good && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+        if (!good) { cudaGetLastError(); return nullptr; }
+        s.ok = true;
+    }
+    return &s;
+}
+
 }  // namespace
 
 extern "C" {
@@ -739,23 +765,36 @@ int invconv_step_host(const float* y_host, const float* w_host, const float* gra
     float* d_gw = (float*)p;    p += wb;
     float* d_ld = (float*)p;
     cudaStream_t st = as_stream(stream);
+    // The copy of grad_x in and the copy of x out run on a side stream: the device has one copy engine per
+    // direction, so x leaves while grad_x arrives and the backward kernels run.  Everything is joined back
+    // into `stream` before the call returns, so the caller still synchronises that stream only.
+    StepSide* side = act_b ? step_side() : nullptr;
+    if (act_b && !side) return INVCONV_CUDA_ERROR;
     cudaMemcpyAsync(d_w, w_host, w_b, cudaMemcpyHostToDevice, st);
     if (act_b) {
+        cudaEventRecord(side->start, st);                     // earlier work on `stream` may still use the scratch
+        cudaStreamWaitEvent(side->side, side->start, 0);
         cudaMemcpyAsync(d_y, y_host, act_b, cudaMemcpyHostToDevice, st);
-        cudaMemcpyAsync(d_gx, grad_x_host, act_b, cudaMemcpyHostToDevice, st);
+        cudaMemcpyAsync(d_gx, grad_x_host, act_b, cudaMemcpyHostToDevice, side->side);
+        cudaEventRecord(side->gx_in, side->side);
     }
     int r = invconv_forward_ws(d_y, d_w, d_x, B, C, H, W, k, ws, ws_b, stream);
     if (r) return r;
+    if (act_b) {
+        cudaEventRecord(side->x_ready, st);
+        cudaStreamWaitEvent(side->side, side->x_ready, 0);
+        cudaMemcpyAsync(x_host, d_x, act_b, cudaMemcpyDeviceToHost, side->side);
+        cudaEventRecord(side->x_out, side->side);
+        cudaStreamWaitEvent(st, side->gx_in, 0);
+    }
     r = invconv_backward_ws(d_gx, d_x, d_w, d_gy, d_gw, B, C, H, W, k, ws, ws_b, stream);
     if (r) return r;
     r = invconv_logdet(d_w, d_ld, C, H, W, k, stream);
     if (r) return r;
-    if (act_b) {
-        cudaMemcpyAsync(x_host, d_x, act_b, cudaMemcpyDeviceToHost, st);
-        cudaMemcpyAsync(grad_y_host, d_gy, act_b, cudaMemcpyDeviceToHost, st);
-    }
+    if (act_b) cudaMemcpyAsync(grad_y_host, d_gy, act_b, cudaMemcpyDeviceToHost, st);
     cudaMemcpyAsync(grad_w_host, d_gw, w_b, cudaMemcpyDeviceToHost, st);
     cudaMemcpyAsync(logdet_host, d_ld, sizeof(float), cudaMemcpyDeviceToHost, st);
+    if (act_b) cudaStreamWaitEvent(st, side->x_out, 0);
     if (cudaGetLastError() != cudaSuccess) return INVCONV_CUDA_ERROR;
     return INVCONV_OK;
 }
