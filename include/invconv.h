@@ -206,7 +206,9 @@ int invconv_get_status(void* stream, int* device_status_out);
  *   mechanism 2: store to a cluster peer's shared memory, cluster barrier, load, one FMA;
  *   mechanism 3: one dependent FMA (the latency of a single accumulator);
  *   mechanism 4: two broadcast 16-byte shared-memory loads feeding 24 FMAs on six accumulators
- *                (one "group" of the wide-channel kernels' inner loop, 8 warps resident).
+ *                (one "group" of the wide-channel kernels' inner loop, 8 warps resident);
+ *   mechanism 5: the arithmetic of one wavefront step for three channels and a 3x3 kernel held in
+ *                registers (six shuffles, 81 FMAs, window rotation; no shared memory).
  * Runs a chain of `steps` dependent steps in one CTA (cluster of 2 for 2) and
  * writes the elapsed SM clock cycles to cycles_out[0] and the chain's final
  * value to cycles_out[1] (device pointer to two 64-bit words).  Used for the

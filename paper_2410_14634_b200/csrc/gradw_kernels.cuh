@@ -255,7 +255,6 @@ __global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(
     // shared-memory set-up needs nothing from the predecessor kernel
     if (tid == 0) { mbar_init(&bar, 1); fence_mbar_init(); }
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 #ifdef INVCONV_GW_TIMING
     long long tg_[8]; tg_[0] = clock64(); tg_[1] = tg_[2] = tg_[5] = tg_[6] = tg_[7] = tg_[0];
 #define GW_TT(i) tg_[i] = clock64()
@@ -350,6 +349,9 @@ __global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(
         }
     }
     GW_TT(2);
+    // let the next kernel on the stream be scheduled only now: its CTAs would otherwise sit on the SMs (and
+    // hold their registers and shared memory) for this kernel's whole run, which measured slower
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // lanes -> warp -> CTA
     {

@@ -23,10 +23,19 @@
 // kernel.  The transposed solve (grad_y, Theorem 1) is the same walk on the
 // image rotated by 180 degrees with  L^-T W_delta^T.
 //
-// grad_w (Theorem 2) is accumulated after the reverse wavefront from the two
-// images still resident in shared memory (grad_y and x): lane = column, rows
-// in order, a k x k window of x in registers; warp partials are combined per
-// CTA and the last CTA to finish sums the CTA partials in a fixed order.
+// grad_w (Theorem 2): up to 81 partial sums ride along in the reverse wavefront
+// (the solved neighbour grad_y[q + delta] is already in registers when x[q] is
+// loaded); warp partials are combined per CTA and the last CTA to finish sums
+// the CTA partials in a fixed order.  Larger kernels and images that stay in
+// global memory get grad_w from the pixel-parallel kernel of gradw_kernels.cuh
+// after the wavefront; a post-pass over the two resident images (lane =
+// column, k x k window of x in registers) remains as the fallback for shapes
+// that kernel's plan does not serve.
+//
+// Two variants of the walk serve shapes where one lane per row is not enough:
+// the ring mode (images larger than shared memory stream through a per-warp
+// ring of 128 columns) and the channel-split walk (lane = row x output
+// channel, for C >= 3 with 5x5 kernels); both are described at their code.
 #pragma once
 
 #include <cstdio>
