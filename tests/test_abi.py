@@ -60,3 +60,33 @@ def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(ImportError):
         binding.lib()
+
+
+def test_dispatch_and_workspace_planning_need_no_device(library):
+    """Host logic only: the family AUTO picks and the scratch a call needs, for the ten benchmark shapes and a
+    few edge shapes (planning falls back to 148 SMs when no device is present)."""
+    from paper_2410_14634_b200 import workloads
+    library.invconv_workspace_bytes.restype = ctypes.c_size_t
+    library.invconv_workspace_bytes.argtypes = [ctypes.c_int] * 5
+    library.invconv_path_for.argtypes = [ctypes.c_int] * 5
+    GENERIC, WARP, TEAM = 1, 2, 3
+    want = {"pr1": WARP, "mnist": WARP, "cifar": WARP, "large64": WARP, "large256": WARP,
+            "cifar_sq": TEAM, "wide48_k3": TEAM, "wide48_k5": TEAM, "wide96_k3": TEAM, "wide96_k5": TEAM}
+    for s in workloads.SHAPES:
+        assert library.invconv_path_for(s.B, s.C, s.H, s.W, s.k) == want[s.name], s.name
+        need = library.invconv_workspace_bytes(s.B, s.C, s.H, s.W, s.k)
+        na = 4 * s.C * s.C * s.k * s.k
+        assert need >= 256 + na, s.name                      # control block + at least one set of partial sums
+        assert need < (64 << 20), s.name
+    # shapes outside the specialised families fall to the generic kernels, which need no scratch
+    assert library.invconv_path_for(1, 3, 8, 8, 7) in (TEAM, GENERIC)
+    assert library.invconv_path_for(1, 128, 64, 64, 3) == GENERIC
+    assert library.invconv_workspace_bytes(1, 128, 64, 64, 3) == 0
+    # invalid shapes report no scratch instead of failing
+    assert library.invconv_workspace_bytes(1, 1, 0, 4, 3) == 0
+    assert library.invconv_workspace_bytes(1, 1, 4, 4, 12) == 0
+    # the scratch of the no-allocation entry point covers every few-channel benchmark shape
+    for s in workloads.SHAPES:
+        if want[s.name] == WARP:
+            assert library.invconv_workspace_bytes(s.B, s.C, s.H, s.W, s.k) <= (1 << 20), s.name
+
