@@ -213,21 +213,31 @@ class _Null:
 
 
 def time_e2e(shape, w, y, gx, device, steps, warmup):
+    """The step through `invconv_step_host` from pinned host buffers, copies inside the timed region.  Two
+    independent sets of host buffers and device scratch alternate on two streams, as an input pipeline would
+    run it, so that one step's copies out overlap the next step's copies in; every step still moves all of
+    its own bytes."""
     import torch
     from paper_2410_14634_b200 import binding
-    hs = binding.HostStep(shape.B, shape.C, shape.H, shape.W, shape.k, device)
-    hs.y.copy_(torch.from_numpy(y)); hs.w.copy_(torch.from_numpy(w)); hs.grad_x.copy_(torch.from_numpy(gx))
-    st = torch.cuda.Stream(device)
-    for _ in range(warmup):
-        hs.run(st)
-    st.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(st)
-    for _ in range(steps):
-        hs.run(st)
-    e1.record(st)
-    st.synchronize()
-    return e0.elapsed_time(e1), hs
+    hss = [binding.HostStep(shape.B, shape.C, shape.H, shape.W, shape.k, device) for _ in range(2)]
+    for hs in hss:
+        hs.y.copy_(torch.from_numpy(y)); hs.w.copy_(torch.from_numpy(w)); hs.grad_x.copy_(torch.from_numpy(gx))
+    sts = [torch.cuda.Stream(device) for _ in range(2)]
+    for i in range(warmup):
+        hss[i & 1].run(sts[i & 1])
+    for st in sts:
+        st.synchronize()
+    e0, e1, ej = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    e0.record(sts[0])
+    sts[1].wait_event(e0)
+    for i in range(steps):
+        hss[i & 1].run(sts[i & 1])
+    ej.record(sts[1])
+    sts[0].wait_event(ej)
+    e1.record(sts[0])
+    for st in sts:
+        st.synchronize()
+    return e0.elapsed_time(e1), hss[0]
 
 
 def cpu_baseline(shape_name, budget_s=12.0):
@@ -312,6 +322,12 @@ def run_ours(args, rank, world):
     value = world * shape.B * args.steps / (ms * 1e-3)
     assert binding.invconv_get_status(device=device) == 0
 
+    # end to end from pinned host memory: every rank runs it at the same time, the slowest rank counts
+    e2e_steps = max(2, min(args.steps, 200))
+    barrier()
+    ms_e, hs = time_e2e(shape, w, y, gx, device, e2e_steps, min(max(args.warmup, 3), 20))
+    ms_e = sharding.max_over_ranks(ms_e, device)
+
     out = None
     if rank == 0:
         # per-kernel durations over the same rotating buffers
@@ -331,8 +347,6 @@ def run_ours(args, rank, world):
         wb = 4 * shape.C * shape.C * shape.k * shape.k
         dom_bytes = 12 * E + 2 * wb
         achieved = dom_bytes / (t_bwd_us * 1e-6) / 1e9
-        e2e_steps = max(1, min(args.steps, 200))
-        ms_e, hs = time_e2e(shape, w, y, gx, device, e2e_steps, min(max(args.warmup, 3), 20))
         cpu = cpu_baseline(args.workload)
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -352,9 +366,10 @@ def run_ours(args, rank, world):
                                     "t_roofline_us": t_roof, "t_achieved_us": t_fwd_us + t_bwd_us,
                                     "frac": t_roof / (t_fwd_us + t_bwd_us)},
             "cpu_baseline": cpu,
-            "e2e": {"value": shape.B * e2e_steps / (ms_e * 1e-3), "unit": UNIT,
+            "e2e": {"value": world * shape.B * e2e_steps / (ms_e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": hs.h2d_bytes, "d2h_bytes_per_step": hs.d2h_bytes,
-                    "ms_per_step": ms_e / e2e_steps, "steps": e2e_steps},
+                    "ms_per_step": ms_e / e2e_steps, "steps": e2e_steps,
+                    "pipeline": "two host-buffer sets alternating on two streams"},
             "gpu_launches": launches,
             "clocks": clocks,
         }

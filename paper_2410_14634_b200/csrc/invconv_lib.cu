@@ -597,6 +597,7 @@ struct StepSide {
     cudaStream_t side = nullptr;
     cudaEvent_t start = nullptr, gx_in = nullptr, x_ready = nullptr, x_out = nullptr;
     bool ok = false;
+    std::mutex enqueue;     // one call at a time records and waits on the events (calls may come from several threads)
 };
 
 StepSide* step_side()
@@ -770,6 +771,8 @@ int invconv_step_host(const float* y_host, const float* w_host, const float* gra
     // into `stream` before the call returns, so the caller still synchronises that stream only.
     StepSide* side = act_b ? step_side() : nullptr;
     if (act_b && !side) return INVCONV_CUDA_ERROR;
+    std::unique_lock<std::mutex> enqueue_lock;
+    if (side) enqueue_lock = std::unique_lock<std::mutex>(side->enqueue);
     cudaMemcpyAsync(d_w, w_host, w_b, cudaMemcpyHostToDevice, st);
     if (act_b) {
         cudaEventRecord(side->start, st);                     // earlier work on `stream` may still use the scratch
