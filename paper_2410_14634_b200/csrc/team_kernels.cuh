@@ -35,21 +35,20 @@ namespace invconv {
 namespace cg = cooperative_groups;
 
 // ---------------------------------------------------------------------------
-// Transformed kernel in two steps:  A[tap][b][a], tap = dh*K + dw,
+// Transformed kernel  A[tap][b][a], tap = dh*K + dw,
 //   forward : tap 0 -> L^-1[a][b];   tap != 0 -> sum_m L^-1[a][m] w[m][b][K-1-dh][K-1-dw]
 //   backward: tap 0 -> L^-1[b][a];   tap != 0 -> sum_m L^-1[m][a] w[b][m][K-1-dh][K-1-dw]
-// L = w[:, :, K-1, K-1] restricted to ci <= co.  L^-1 is built by blocked
-// recursion: 12x12 diagonal blocks by column-parallel substitution, then pairs
-// of blocks are merged,  [[X11, 0], [-X22 L21 X11, X22]],  doubling the block
-// size each level, so the depth is logarithmic in C.
-// Shared memory: three C x C matrices (rows padded to 16 bytes).
-// ---------------------------------------------------------------------------
-// One CTA per input channel b (plus one for tap 0) solves  T S = RHS  by right-looking substitution in shared
-// memory, T = L (forward, rows ascending) or L^T (backward, rows descending):
+// L = w[:, :, K-1, K-1] restricted to ci <= co.
+// One CTA per input channel b (plus CTAs for tap 0) solves  T S = RHS  by blocked right-looking substitution
+// in shared memory, T = L (forward, rows ascending) or L^T (backward, rows descending):
 //   b <  C : RHS[m][kk] = w[m][b][kk] (forward) / w[b][m][kk] (backward); S[a][kk] -> A[flip(kk)][b][a]
 //   b >= C : RHS = 32 columns of the identity;                            S[a][b'] -> A[0][b'][a]
-// Step a scales nothing in place: every update of a later row i reads the finished row a and its diagonal,
-//   RHS[i][:] -= T[i][a] * RHS[a][:] / T[a][a],   one block barrier per row.
+// Pivot blocks of eight rows: every thread (row lane, column) first solves the block's 8x8 triangle for its
+// column in registers (redundantly across row lanes: 28 FMAs), then subtracts the block's contribution from
+// its share of the rows behind the block -- one block barrier per eight rows instead of one per row (the
+// barrier and its shared-memory round trip were the cost: 0.4 us per row at C = 48).  Solved rows go to a
+// separate array so that no thread reads a row another thread is rewriting.
+// ---------------------------------------------------------------------------
 template <bool BWD>
 __global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K)
 {
@@ -63,7 +62,8 @@ __global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict
     const int NC = ident ? min(32, C - c0) : KK;   // right-hand-side columns
     float* L = sm;                            // [C][C]  L[i][j], j <= i
     float* invd = sm + C * C;                 // [C]
-    float* RHS = invd + ((C + 3) & ~3);       // [C][NC]
+    float* RHS = invd + ((C + 3) & ~3);       // [C][NC]  residuals
+    float* Y = RHS + C * (KK > 32 ? KK : 32); // [C][NC]  solved rows
 
     for (int e0 = tid; e0 < C * C; e0 += NT * 8) {
         float tv[8];
@@ -104,32 +104,53 @@ __global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict
     }
     __syncthreads();
     // thread = (row lane ty, column tx): no divisions inside the substitution loop
+    constexpr int NBK = 8;
     const int NCP = NC <= 32 ? 32 : NC;
     const int tx = tid % NCP, ty = tid / NCP, TY = NT / NCP;
-    for (int st = 0; st < C - 1; ++st) {
-        const int a = BWD ? C - 1 - st : st;
-        const int nrest = C - 1 - st;                     // rows still to update
-        const float da = invd[a];
+    auto idx = [&](int pos) { return BWD ? C - 1 - pos : pos; };              // position in solve order -> row index
+    auto tval = [&](int pi, int pa) {                                          // T[row at pi][row at pa], pi behind pa
+        const int i = idx(pi), a = idx(pa);
+        return BWD ? L[a * C + i] : L[i * C + a];
+    };
+    for (int b0 = 0; b0 < C; b0 += NBK) {
+        const int nb = min(NBK, C - b0);
         if (tx < NC && ty < TY) {
-            const float ra = -da * RHS[a * NC + tx];
-#pragma unroll 4
+            float rr[NBK], yy[NBK];
+#pragma unroll
+            for (int q = 0; q < NBK; ++q) rr[q] = q < nb ? RHS[idx(b0 + q) * NC + tx] : 0.f;
+#pragma unroll
+            for (int q = 0; q < NBK; ++q) {
+                yy[q] = q < nb ? rr[q] * invd[idx(b0 + (q < nb ? q : 0))] : 0.f;
+#pragma unroll
+                for (int q2 = q + 1; q2 < NBK; ++q2)
+                    if (q2 < nb) rr[q2] = fmaf(-tval(b0 + q2, b0 + q), yy[q], rr[q2]);
+            }
+            if (ty == 0) {
+#pragma unroll
+                for (int q = 0; q < NBK; ++q)
+                    if (q < nb) Y[idx(b0 + q) * NC + tx] = yy[q];
+            }
+            const int nrest = C - (b0 + nb);                                   // rows behind the block
             for (int ri = ty; ri < nrest; ri += TY) {
-                const int i = BWD ? a - 1 - ri : a + 1 + ri;
-                const float t = BWD ? L[a * C + i] : L[i * C + a];      // T[i][a]
-                RHS[i * NC + tx] = fmaf(t, ra, RHS[i * NC + tx]);
+                const int pi = b0 + nb + ri, i = idx(pi);
+                float acc = RHS[i * NC + tx];
+#pragma unroll
+                for (int q = 0; q < NBK; ++q)
+                    if (q < nb) acc = fmaf(-tval(pi, b0 + q), yy[q], acc);
+                RHS[i * NC + tx] = acc;
             }
         }
         __syncthreads();
     }
     for (int e = tid; e < C * NC; e += NT) {
         const int col = e / C, a = e - col * C;               // a fastest: coalesced stores
-        const float v = RHS[a * NC + col] * invd[a];
+        const float v = Y[a * NC + col];
         if (ident) A[(size_t)(c0 + col) * C + a] = v;         // A[0][b' = c0 + col][a]
         else if (col != ctr) A[((size_t)(KK - 1 - col) * C + b) * C + a] = v;
     }
 }
 
-inline size_t team_solve_smem(int C, int K) { return sizeof(float) * ((size_t)C * C + ((C + 3) & ~3) + (size_t)C * (K * K > 32 ? K * K : 32)); }
+inline size_t team_solve_smem(int C, int K) { return sizeof(float) * ((size_t)C * C + ((C + 3) & ~3) + 2 * (size_t)C * (K * K > 32 ? K * K : 32)); }
 
 // ---------------------------------------------------------------------------
 struct TeamParams {
