@@ -129,6 +129,132 @@ __global__ void __launch_bounds__(256) gradw_tile_kernel(GradWParams p)
         }
 }
 
+// ---------------------------------------------------------------------------
+// The same tiling on the tensor pipe (TF32 inputs, fp32 accumulation): for a
+// fixed tap the sum over pixels is a matrix product  G[co][ci] = sum_p
+// grad_y[co][p] * x[ci][p - shift], M = co, N = ci, contraction over the
+// pixels, which are the contiguous index of both operands in NCHW.  A warp
+// owns one 16-row block of output channels and one kernel column dw and walks
+// the rows h >= dh of the staged planes in chunks of eight pixels:
+// mma.m16n8k8 with A = grad_y[16 co][8 pixels], B = x[8 pixels - shift][8 ci]
+// for each of the tile's 8-channel groups.  Fragments are read straight from
+// the padded channel planes (plane stride = 4 mod 32: the 8 x 4 elements of a
+// fragment register fall in 32 different banks); the K-1 pixels to the left of
+// column 0 and the rows above row 0 are zeros by predicate.  Inputs are
+// rounded to TF32 (10-bit mantissa): the weight gradient's parity bar is 1e-3
+// of its largest entry, which a single TF32 pass holds (the solves, at 1e-4,
+// stay in fp32).  Needs W % 8 == 0; other shapes use the FMA kernel above.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ unsigned to_tf32(float v)
+{
+    unsigned r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+    return r;
+}
+
+__device__ __forceinline__ void mma_tf32_16x8x8(float (&d)[4], const unsigned (&a)[4], const unsigned (&b)[2])
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+template <int TC, int K>
+__global__ void __launch_bounds__(32 * TC * K) gradw_mma_kernel(GradWParams p)
+{
+    extern __shared__ __align__(128) float smem[];
+    constexpr int TB = 16 * TC;                 // channels per tile side
+    constexpr int NT8 = 2 * TC;                 // 8-channel groups of the ci tile
+    const int H = p.H, W = p.W, HW = H * W, C = p.C;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
+    const int g = lane >> 2, t = lane & 3;      // fragment coordinates
+    const int mt = warp / K, dw = warp - mt * K; // this warp's 16 output channels and kernel column
+    int bid = blockIdx.x;
+    const int share = bid % p.nbc; bid /= p.nbc;
+    const int tci = bid % p.tiles; bid /= p.tiles;
+    const int tco = bid % p.tiles; bid /= p.tiles;
+    const int dh = bid;
+    const int co0 = tco * TB, ci0 = tci * TB;
+    const int nco = min(TB, C - co0), nci = min(TB, C - ci0);
+    float* gys = smem;                          // [TB][plane]
+    float* xs = smem + TB * p.plane;            // [TB][plane]
+
+    float acc[NT8][4];
+#pragma unroll
+    for (int i = 0; i < NT8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+#ifdef INVCONV_GW_TIMING
+    long long tm_[5]; tm_[0] = clock64(); tm_[1] = tm_[2] = tm_[0];
+#endif
+    // channels beyond C (padding of the last tile) stay zero; the others are overwritten by every image
+    for (int c = nco + warp; c < TB; c += nwarps)
+        for (int i = lane; i < p.plane; i += 32) gys[c * p.plane + i] = 0.f;
+    for (int c = nci + warp; c < TB; c += nwarps)
+        for (int i = lane; i < p.plane; i += 32) xs[c * p.plane + i] = 0.f;
+
+    for (int n = share; n < p.B; n += p.nbc) {
+        // stage the tile's channel planes with 16-byte asynchronous copies issued by all threads (a bulk copy
+        // per channel plane would serialise in the copy engine at ~150 cycles each, more than the whole product)
+        const float* gsrc = p.gy + ((size_t)n * C + co0) * HW;
+        const float* xsrc = p.x + ((size_t)n * C + ci0) * HW;
+        const int nq = HW >> 2;
+        for (int c = warp; c < nco + nci; c += nwarps) {
+            const bool isg = c < nco;
+            const int cc = isg ? c : c - nco;
+            const float* src = (isg ? gsrc : xsrc) + (size_t)cc * HW;
+            float* dstp = (isg ? gys : xs) + cc * p.plane;
+            for (int q = lane; q < nq; q += 32) cp_async_f32x4(dstp + 4 * q, src + 4 * q, true);
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+#ifdef INVCONV_GW_TIMING
+        tm_[1] = clock64();
+#endif
+
+        const float* ga = gys + (mt * 16 + g) * p.plane + t;          // A: rows g and g + 8, pixel columns t and t + 4
+        const float* xb = xs + g * p.plane + t - dw;                  // B: channel g of a group, pixels t and t + 4, shifted
+        for (int h = dh; h < H; ++h) {
+            for (int w0 = 0; w0 < W; w0 += 8) {
+                const int pa = h * W + w0, pb = (h - dh) * W + w0;
+                unsigned a[4];
+                a[0] = to_tf32(ga[pa]);
+                a[1] = to_tf32(ga[pa + 8 * p.plane]);
+                a[2] = to_tf32(ga[pa + 4]);
+                a[3] = to_tf32(ga[pa + 8 * p.plane + 4]);
+                const bool v0 = w0 + t >= dw, v1 = w0 + t + 4 >= dw;   // pixels left of column 0 are padding
+#pragma unroll
+                for (int nt = 0; nt < NT8; ++nt) {
+                    unsigned b[2];
+                    b[0] = v0 ? to_tf32(xb[nt * 8 * p.plane + pb]) : 0u;
+                    b[1] = v1 ? to_tf32(xb[nt * 8 * p.plane + pb + 4]) : 0u;
+                    mma_tf32_16x8x8(acc[nt], a, b);
+                }
+            }
+        }
+#ifdef INVCONV_GW_TIMING
+        tm_[2] = clock64();
+#endif
+        __syncthreads();       // everyone is done with this image before its planes are overwritten
+    }
+
+    float* dst = p.partials + (size_t)share * K * K * C * C + (size_t)(dh * K + dw) * C * C;
+#pragma unroll
+    for (int nt = 0; nt < NT8; ++nt)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int co = co0 + mt * 16 + g + (j >> 1) * 8, ci = ci0 + nt * 8 + 2 * t + (j & 1);
+            if (co < C && ci < C) dst[(size_t)co * C + ci] = acc[nt][j];
+        }
+#ifdef INVCONV_GW_TIMING
+    tm_[3] = clock64();
+    if (tid == 0 && blockIdx.x == 0)
+        printf("gradw_mma (cycles) block 0: staged %lld | computed %lld | written %lld\n", tm_[1] - tm_[0], tm_[2] - tm_[0], tm_[3] - tm_[0]);
+#endif
+}
+
 // grad_w[co][ci][K-1-dh][K-1-dw] = -(sum over shares), zero outside the channel mask of the centre tap.
 __global__ void __launch_bounds__(256) gradw_reduce_kernel(const float* __restrict__ partials, float* __restrict__ grad_w,
                                                            int nbc, int C, int K)

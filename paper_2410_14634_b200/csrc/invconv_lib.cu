@@ -389,6 +389,16 @@ int launch_gradw_inst(const GradWPlan& gp, const GradWParams& prm, cudaStream_t 
     return check_launch();
 }
 
+template <int TC, int K>
+int launch_gradw_mma_inst(const GradWPlan& gp, const GradWParams& prm, cudaStream_t st)
+{
+    auto kern = gradw_mma_kernel<TC, K>;
+    const int rc = set_smem_limit(kern, gp.smem);
+    if (rc) return rc;
+    kern<<<gp.grid, 32 * TC * K, gp.smem, st>>>(prm);
+    return check_launch();
+}
+
 // grad_w through the tiled correlation kernel; partial sums live behind the transformed kernel in the workspace.
 int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, cudaStream_t st)
 {
@@ -404,7 +414,13 @@ int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, c
     prm.partials = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES) + na + (size_t)g.C * g.C;
     prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W; prm.nbc = gp.nbc; prm.tiles = gp.tiles; prm.plane = gp.plane;
     int rc = INVCONV_UNSUPPORTED;
-#define X(TT, KK_) if (gp.TC == TT && g.k == KK_) rc = launch_gradw_inst<TT, KK_>(gp, prm, st);
+    // tensor pipe (TF32 inputs) where the fragments line up: rows of whole 8-pixel chunks, conflict-free planes
+    const char* knob = std::getenv("INVCONV_GW_MMA");
+    // (measured: 31 / 58 us against 41 / 87 us for the FMA kernel on the 48-channel shapes, k = 3 / 5; no gain
+    // for tiles of 16 channels, which keep the FMA kernel)
+    const bool mma = gp.TC == 3 && g.W % 8 == 0 && gp.plane % 32 == 4 && !(knob && knob[0] == '0');
+#define X(TT, KK_)                                                                                    \
+    if (gp.TC == TT && g.k == KK_) rc = mma ? launch_gradw_mma_inst<TT, KK_>(gp, prm, st) : launch_gradw_inst<TT, KK_>(gp, prm, st);
     X(1, 1) X(1, 2) X(1, 3) X(1, 5) X(3, 1) X(3, 2) X(3, 3) X(3, 5)
 #undef X
     if (rc) return rc;

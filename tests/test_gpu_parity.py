@@ -224,6 +224,27 @@ def test_training_step_calls_with_the_log_det_folded_in(B, oracle, shape):
     assert nmax_err(d, gl * oracle.logdet_grad_w(w, H, W)) <= 1e-5
 
 
+@pytest.mark.parametrize("mma", ["0", "1"])
+@pytest.mark.parametrize("shape", [(3, 48, 8, 8, 3), (2, 40, 6, 16, 2), (2, 33, 16, 16, 5), (5, 96, 8, 8, 3)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_grad_w_many_channels_fma_and_tensor_pipe(B, oracle, shape, mma, monkeypatch):
+    """grad_w at many channels through the FMA tile kernel and through the TF32 tensor-pipe kernel (channel
+    counts off the tile size, several images per batch share): both inside the 1e-3 bar; the FMA kernel, which
+    keeps fp32 inputs, far inside it."""
+    monkeypatch.setenv("INVCONV_GW_MMA", mma)
+    Bn, C, H, W, k = shape
+    w, y, gx = workloads.make_custom(700 + sum(shape), Bn, C, H, W, k, sigma=0.05 / np.sqrt(C))
+    x_ref = oracle.invconv_forward(y, w)
+    gy_ref, gw_ref = oracle.invconv_backward(gx, x_ref, w)
+    B.invconv_set_path(PATHS["team"])
+    try:
+        _, gw = run_or_skip(B, B.invconv_backward, dev(gx), dev(x_ref.astype(np.float32)), dev(w))
+    finally:
+        B.invconv_set_path(0)
+    err = nmax_err(gw.cpu().numpy(), gw_ref)
+    assert err <= (TOL_GW if mma == "1" else 2e-5), err
+
+
 def test_empty_batch_is_a_no_op_and_zeroes_grad_w(B):
     import torch
     w = dev(workloads.make_custom(9, 1, 2, 4, 4, 3)[0])
