@@ -256,23 +256,41 @@ __global__ void __launch_bounds__(32 * TC * K) gradw_mma_kernel(GradWParams p)
 }
 
 // grad_w[co][ci][K-1-dh][K-1-dw] = -(sum over shares), zero outside the channel mask of the centre tap.
+// LANES adjacent lanes share one entry: lane q adds the shares b = q, q+LANES, ... in that order (up to sixteen
+// loads in flight), then the LANES sums are combined in a fixed order by shuffles -- the result does not depend
+// on scheduling.  LANES = 4 shortens the chain of dependent loads where there are few entries (few CTAs);
+// LANES = 1 (one thread per entry, fully coalesced rows) is faster where the entries alone fill the GPU.
+template <int LANES>
 __global__ void __launch_bounds__(256) gradw_reduce_kernel(const float* __restrict__ partials, float* __restrict__ grad_w,
                                                            int nbc, int C, int K)
 {
+    constexpr int EPW = 32 / LANES;                      // entries per warp
+    constexpr int INF = LANES == 1 ? 8 : 16;             // loads in flight per thread
     const int NA = K * K * C * C;
-    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < NA; e += gridDim.x * blockDim.x) {
+    const int q = threadIdx.x % LANES;
+    const int nper = (nbc + LANES - 1) / LANES;          // shares per lane
+    const int NAR = (NA + EPW - 1) / EPW * EPW;          // whole warps stay in the loop for the shuffles
+    for (int e0 = (blockIdx.x * blockDim.x + threadIdx.x) / LANES; e0 < NAR; e0 += (gridDim.x * blockDim.x) / LANES) {
+        const int e = e0 < NA ? e0 : NA - 1;
         float s = 0.f;
-        for (int b0 = 0; b0 < nbc; b0 += 8) {              // eight loads in flight; the sum stays in share order
-            float v[8];
+        for (int i0 = 0; i0 < nper; i0 += INF) {
+            float v[INF];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = __ldcg(partials + (size_t)min(b0 + q, nbc - 1) * NA + e);
+            for (int j = 0; j < INF; ++j) {
+                const int b = q + LANES * (i0 + j);
+                v[j] = __ldcg(partials + (size_t)(b < nbc ? b : nbc - 1) * NA + e);
+            }
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-                if (b0 + q < nbc) s += v[q];
+            for (int j = 0; j < INF; ++j)
+                if (q + LANES * (i0 + j) < nbc) s += v[j];
         }
-        const int ci = e % C, co = (e / C) % C, tap = e / (C * C);
-        const int dh = tap / K, dw = tap % K;
-        grad_w[((co * C + ci) * K + (K - 1 - dh)) * K + (K - 1 - dw)] = (tap == 0 && ci > co) ? 0.f : -s;
+#pragma unroll
+        for (int o = 1; o < LANES; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (q == 0 && e0 < NA) {
+            const int ci = e % C, co = (e / C) % C, tap = e / (C * C);
+            const int dh = tap / K, dw = tap % K;
+            grad_w[((co * C + ci) * K + (K - 1 - dh)) * K + (K - 1 - dw)] = (tap == 0 && ci > co) ? 0.f : -s;
+        }
     }
 }
 

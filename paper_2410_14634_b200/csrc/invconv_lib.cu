@@ -424,8 +424,12 @@ int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, c
     X(1, 1) X(1, 2) X(1, 3) X(1, 5) X(3, 1) X(3, 2) X(3, 3) X(3, 5)
 #undef X
     if (rc) return rc;
-    const int blocks = (int)((na + 255) / 256 < 4096 ? (na + 255) / 256 : 4096);
-    gradw_reduce_kernel<<<blocks, 256, 0, st>>>(prm.partials, gw, gp.nbc, g.C, g.k);
+    if (na < 16384) {       // few entries: four lanes per entry (64 entries per CTA)
+        gradw_reduce_kernel<4><<<(int)((na + 63) / 64), 256, 0, st>>>(prm.partials, gw, gp.nbc, g.C, g.k);
+    } else {
+        const int blocks = (int)((na + 255) / 256 < 4096 ? (na + 255) / 256 : 4096);
+        gradw_reduce_kernel<1><<<blocks, 256, 0, st>>>(prm.partials, gw, gp.nbc, g.C, g.k);
+    }
     return check_launch();
 }
 
