@@ -159,21 +159,25 @@ __device__ __forceinline__ void mma_tf32_16x8x8(float (&d)[4], const unsigned (&
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
 
-template <int TC, int K>
-__global__ void __launch_bounds__(32 * TC * K) gradw_mma_kernel(GradWParams p)
+// ALLDH (tiles of 16 channels): one CTA covers all K*K taps, warp = (dh, dw), so that a 12- or 16-channel
+// layer still gives every CTA K*K warps and every image is staged once instead of once per kernel row.
+template <int TC, int K, bool ALLDH = false>
+__global__ void __launch_bounds__(32 * (ALLDH ? K * K : TC * K)) gradw_mma_kernel(GradWParams p)
 {
+    static_assert(!ALLDH || TC == 1, "all kernel rows in one CTA: tiles of 16 channels only");
     extern __shared__ __align__(128) float smem[];
     constexpr int TB = 16 * TC;                 // channels per tile side
     constexpr int NT8 = 2 * TC;                 // 8-channel groups of the ci tile
     const int H = p.H, W = p.W, HW = H * W, C = p.C;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
     const int g = lane >> 2, t = lane & 3;      // fragment coordinates
-    const int mt = warp / K, dw = warp - mt * K; // this warp's 16 output channels and kernel column
+    const int mt = ALLDH ? 0 : warp / K;        // this warp's 16 output channels
+    const int dw = ALLDH ? warp % K : warp - mt * K;   // ... and kernel column
     int bid = blockIdx.x;
     const int share = bid % p.nbc; bid /= p.nbc;
     const int tci = bid % p.tiles; bid /= p.tiles;
     const int tco = bid % p.tiles; bid /= p.tiles;
-    const int dh = bid;
+    const int dh = ALLDH ? warp / K : bid;
     const int co0 = tco * TB, ci0 = tci * TB;
     const int nco = min(TB, C - co0), nci = min(TB, C - ci0);
     float* gys = smem;                          // [TB][plane]
@@ -297,6 +301,7 @@ __global__ void __launch_bounds__(256) gradw_reduce_kernel(const float* __restri
 struct GradWPlan {
     bool ok = false;
     int TC = 3, tiles = 1, nbc = 1, plane = 0, grid = 0;
+    int nbc_all = 0, grid_all = 0;      // tiles of 16 channels on the tensor pipe: shares and CTAs when one CTA covers all taps
     size_t smem = 0;
 };
 
@@ -326,6 +331,15 @@ inline GradWPlan plan_gradw(int B, int C, int H, int W, int K, size_t max_smem, 
     nbc = (B + per - 1) / per;
     pl.nbc = nbc;
     pl.grid = K * pl.tiles * pl.tiles * nbc;
+    if (pl.TC == 1) {
+        int na = (2 * sm_count) / (pl.tiles * pl.tiles);
+        if (na < 1) na = 1;
+        if (na > B) na = B;
+        const int pa = (B + na - 1) / na;
+        na = (B + pa - 1) / pa;
+        pl.nbc_all = na;
+        pl.grid_all = pl.tiles * pl.tiles * na;
+    }
     pl.ok = true;
     return pl;
 }

@@ -376,7 +376,8 @@ size_t team_workspace_bytes(int B, int C, int H, int W, int k)
     if (!team_plan(B, C, H, W, k).ok) return 0;
     const size_t na = sizeof(float) * (size_t)k * k * C * C;
     const GradWPlan gp = gradw_plan(B, C, H, W, k);
-    return INVCONV_WS_CONTROL_BYTES + na + sizeof(float) * (size_t)C * C + (gp.ok ? na * gp.nbc : 0);
+    const int shares = gp.nbc > gp.nbc_all ? gp.nbc : gp.nbc_all;
+    return INVCONV_WS_CONTROL_BYTES + na + sizeof(float) * (size_t)C * C + (gp.ok ? na * shares : 0);
 }
 
 template <int TC, int K>
@@ -399,6 +400,16 @@ int launch_gradw_mma_inst(const GradWPlan& gp, const GradWParams& prm, cudaStrea
     return check_launch();
 }
 
+template <int K>
+int launch_gradw_mma_all_inst(const GradWPlan& gp, const GradWParams& prm, cudaStream_t st)
+{
+    auto kern = gradw_mma_kernel<1, K, true>;
+    const int rc = set_smem_limit(kern, gp.smem);
+    if (rc) return rc;
+    kern<<<gp.grid_all, 32 * K * K, gp.smem, st>>>(prm);
+    return check_launch();
+}
+
 // grad_w through the tiled correlation kernel; partial sums live behind the transformed kernel in the workspace.
 int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, cudaStream_t st)
 {
@@ -416,19 +427,29 @@ int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, c
     int rc = INVCONV_UNSUPPORTED;
     // tensor pipe (TF32 inputs) where the fragments line up: rows of whole 8-pixel chunks, conflict-free planes
     const char* knob = std::getenv("INVCONV_GW_MMA");
-    // (measured: 31 / 58 us against 41 / 87 us for the FMA kernel on the 48-channel shapes, k = 3 / 5; no gain
-    // for tiles of 16 channels, which keep the FMA kernel)
-    const bool mma = gp.TC == 3 && g.W % 8 == 0 && gp.plane % 32 == 4 && !(knob && knob[0] == '0');
+    // (measured, kernel + reduction: 31 / 58 us against 41 / 87 us for the FMA kernel on the 48-channel shapes,
+    // k = 3 / 5; 19 us against 25 us on the 12-channel one with all taps in one CTA)
+    const bool mma = g.W % 8 == 0 && gp.plane % 32 == 4 && !(knob && knob[0] == '0');
+    int shares = gp.nbc;
+    if (mma && gp.TC == 1) {                 // tiles of 16 channels: one CTA covers all taps, its own share count
+        shares = gp.nbc_all;
+        prm.nbc = shares;
+        if (g.k == 1) rc = launch_gradw_mma_all_inst<1>(gp, prm, st);
+        if (g.k == 2) rc = launch_gradw_mma_all_inst<2>(gp, prm, st);
+        if (g.k == 3) rc = launch_gradw_mma_all_inst<3>(gp, prm, st);
+        if (g.k == 5) rc = launch_gradw_mma_all_inst<5>(gp, prm, st);
+    } else {
 #define X(TT, KK_)                                                                                    \
-    if (gp.TC == TT && g.k == KK_) rc = mma ? launch_gradw_mma_inst<TT, KK_>(gp, prm, st) : launch_gradw_inst<TT, KK_>(gp, prm, st);
+    if (gp.TC == TT && g.k == KK_) rc = (mma && TT == 3) ? launch_gradw_mma_inst<TT, KK_>(gp, prm, st) : launch_gradw_inst<TT, KK_>(gp, prm, st);
     X(1, 1) X(1, 2) X(1, 3) X(1, 5) X(3, 1) X(3, 2) X(3, 3) X(3, 5)
 #undef X
+    }
     if (rc) return rc;
     if (na < 16384) {       // few entries: four lanes per entry (64 entries per CTA)
-        gradw_reduce_kernel<4><<<(int)((na + 63) / 64), 256, 0, st>>>(prm.partials, gw, gp.nbc, g.C, g.k);
+        gradw_reduce_kernel<4><<<(int)((na + 63) / 64), 256, 0, st>>>(prm.partials, gw, shares, g.C, g.k);
     } else {
         const int blocks = (int)((na + 255) / 256 < 4096 ? (na + 255) / 256 : 4096);
-        gradw_reduce_kernel<1><<<blocks, 256, 0, st>>>(prm.partials, gw, gp.nbc, g.C, g.k);
+        gradw_reduce_kernel<1><<<blocks, 256, 0, st>>>(prm.partials, gw, shares, g.C, g.k);
     }
     return check_launch();
 }
