@@ -483,9 +483,20 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
                 for (int i = finq_i0, aq = finq_a0; i < npix; ) {
                     const float* src2 = red + (size_t)i * NWP * CAp + aq * 4;
                     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int ww = 0; ww < NWP; ++ww) {
-                        const float4 t4 = *reinterpret_cast<const float4*>(src2 + ww * CAp);
-                        v.x += t4.x; v.y += t4.y; v.z += t4.z; v.w += t4.w;
+                    if constexpr (NGN <= 6) {
+                        // all warps' partial sums in flight at once (NWP <= 8); the variants that hold more taps
+                        // per thread have no registers to spare for this and measured slower with it
+                        float4 tv[8];
+#pragma unroll
+                        for (int ww = 0; ww < 8; ++ww)
+                            tv[ww] = ww < NWP ? *reinterpret_cast<const float4*>(src2 + ww * CAp) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                        for (int ww = 0; ww < 8; ++ww) { v.x += tv[ww].x; v.y += tv[ww].y; v.z += tv[ww].z; v.w += tv[ww].w; }
+                    } else {
+                        for (int ww = 0; ww < NWP; ++ww) {
+                            const float4 t4 = *reinterpret_cast<const float4*>(src2 + ww * CAp);
+                            v.x += t4.x; v.y += t4.y; v.z += t4.z; v.w += t4.w;
+                        }
                     }
                     const int o = obase + i * DS + aq * 4;
                     *reinterpret_cast<float4*>(U + o) = v;
