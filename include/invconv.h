@@ -58,7 +58,8 @@ enum invconv_path {
     INVCONV_PATH_AUTO = 0,
     INVCONV_PATH_GENERIC = 1,     /* one CTA per image, operands in global memory, any shape */
     INVCONV_PATH_WARP = 2,        /* warp-shuffle wavefront, image resident in shared memory, small C */
-    INVCONV_PATH_TEAM = 3         /* CTA / cluster per image, register-tiled channel contraction, wide C */
+    INVCONV_PATH_TEAM = 3,        /* CTA / cluster per image, register-tiled channel contraction, wide C */
+    INVCONV_PATH_TENSOR = 4       /* cluster per group of images, channel contraction on the tcgen05 tensor cores */
 };
 
 /* x = f^{-1}(y): the inverse of the masked convolution, by wavefront

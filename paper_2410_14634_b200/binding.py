@@ -17,7 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libinvconv_b200.so")
 
 OK, BAD_ARG, UNSUPPORTED, CUDA_ERROR, TIMEOUT, WORKSPACE_TOO_SMALL = range(6)
-PATH_AUTO, PATH_GENERIC, PATH_WARP, PATH_TEAM = range(4)
+PATH_AUTO, PATH_GENERIC, PATH_WARP, PATH_TEAM, PATH_TENSOR = range(5)
 WS_CONTROL_BYTES = 256
 
 _lib = None

@@ -25,18 +25,53 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def _includes(path: str, seen: set) -> set:
+    """Files reachable from `path` through #include "..." (searched in csrc/ and include/)."""
+    if path in seen:
+        return seen
+    seen.add(path)
+    with open(path) as fh:
+        for line in fh:
+            line = line.strip()
+            if line.startswith('#include "'):
+                name = line.split('"')[1]
+                for d in (CSRC, os.path.join(ROOT, "include")):
+                    cand = os.path.join(d, name)
+                    if os.path.exists(cand):
+                        _includes(cand, seen)
+    return seen
+
+
+def _object_stale(obj: str, src: str) -> bool:
+    if not os.path.exists(obj):
+        return True
+    t = os.path.getmtime(obj)
+    return any(os.path.getmtime(d) > t for d in _includes(src, set()))
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile csrc/*.cu into libinvconv_b200.so next to this file."""
+    """Compile every csrc/*.cu (one object each, in parallel) and link libinvconv_b200.so next to this file."""
     if not force and not _stale():
         return LIB
-    tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [NVCC, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-           "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    objdir = os.path.join(PKG, "build")
+    os.makedirs(objdir, exist_ok=True)
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
+             "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("INVCONV_NVCC_FLAGS", "").split()      # e.g. -DINVCONV_TEAM_TIMING for development builds
-    cmd += sources() + ["-o", tmp]
-    subprocess.check_call(cmd)
+        flags += ["-Xptxas", "-v"]
+    extra = os.environ.get("INVCONV_NVCC_FLAGS", "").split()     # development builds only
+    flags += extra
+    procs, objs = [], []
+    for src in sources():
+        obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
+        objs.append(obj)
+        if force or extra or _object_stale(obj, src):
+            procs.append((src, subprocess.Popen([NVCC, "-c", *flags, src, "-o", obj])))
+    failed = [src for src, pr in procs if pr.wait() != 0]
+    if failed:
+        raise RuntimeError(f"nvcc failed for {failed}")
+    tmp = LIB + f".tmp{os.getpid()}"
+    subprocess.check_call([NVCC, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-Xcompiler", "-fPIC", *objs, "-o", tmp])
     os.replace(tmp, LIB)
     return LIB
 

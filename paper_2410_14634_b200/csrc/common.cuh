@@ -13,9 +13,9 @@ struct Geom {
     int B, C, H, W, k;
 };
 
-// Device-side status word (one per device that loads the library).  Kernels
-// only ever raise it (atomicMax) when a bounded wait gives up.
-__device__ int g_device_status = 0;
+// Device-side status word (one per device that loads the library and per translation unit).  Kernels
+// only ever raise it (atomicMax) when a bounded wait gives up; invconv_get_status reads every copy.
+static __device__ int g_device_status = 0;
 
 __device__ __forceinline__ void raise_status(int code) { atomicMax(&g_device_status, code); }
 
@@ -25,6 +25,14 @@ __host__ __device__ __forceinline__ size_t act_index(int n, int c, int h, int w,
 }
 __host__ __device__ __forceinline__ int w_index(int co, int ci, int a, int b, int C, int k) {
     return ((co * C + ci) * k + a) * k + b;
+}
+
+// Round to nearest tf32 (10 explicit mantissa bits; the low 13 bits of the result are zero).
+__device__ __forceinline__ float tf32_hi(float v)
+{
+    uint32_t u;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(v));
+    return __uint_as_float(u);
 }
 
 // Upper bound on polls of any device-side wait before it gives up.

@@ -16,10 +16,14 @@
 #include "probe_kernels.cuh"
 #include "warp_kernels.cuh"
 #include "team_kernels.cuh"
+#include "tensor_plan.h"
+#include "lib_internal.h"
 #include "gradw_kernels.cuh"
 #include "conv_kernels.cuh"
 
 using namespace invconv;
+using invconv_internal::set_smem_limit;
+using invconv_internal::kMaxDynSmem;
 
 namespace {
 
@@ -29,6 +33,9 @@ std::atomic<bool> g_use_pdl{std::getenv("INVCONV_NO_PDL") == nullptr};   // meas
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
+}  // namespace
+
+namespace invconv_internal {
 // Called once after every kernel launch of the library.
 int check_launch()
 {
@@ -40,6 +47,10 @@ int check_launch()
     }
     return INVCONV_OK;
 }
+}  // namespace invconv_internal
+using invconv_internal::check_launch;
+
+namespace {
 
 int check_shape(int B, int C, int H, int W, int k)
 {
@@ -50,7 +61,6 @@ int check_shape(int B, int C, int H, int W, int k)
     return INVCONV_OK;
 }
 
-constexpr size_t kMaxDynSmem = 226 * 1024;   // 227 KiB per CTA minus the kernels' static shared memory
 
 // ---------------------------------------------------------------- warp family
 #define INVCONV_WARP_CASES(X) \
@@ -115,17 +125,6 @@ WarpPlan plan_warp(int B, int C, int H, int W, int k, bool bwd)
     return WarpPlan{};
 }
 
-template <typename Kern>
-int set_smem_limit(Kern kern, size_t smem)
-{
-    if (smem <= 48 * 1024) return INVCONV_OK;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-        cudaGetLastError();
-        return INVCONV_CUDA_ERROR;
-    }
-    return INVCONV_OK;
-}
-
 template <int C, int K, bool BWD>
 int launch_warp_ck(const WarpPlan& pl, WarpParams prm, cudaStream_t st)
 {
@@ -171,7 +170,7 @@ int launch_warp_ck(const WarpPlan& pl, WarpParams prm, cudaStream_t st)
 
 constexpr size_t kGradWSmallSmem = 96 * 1024;
 
-int sm_count();
+using invconv_internal::sm_count;
 
 GradWSmallPlan gradw_small_plan(int B, int C, int H, int W, int k)
 {
@@ -346,19 +345,24 @@ int launch_masked_conv_small(const float* x, const float* w, float* y, Geom g, c
 }
 
 // ---------------------------------------------------------------- team family
+}  // namespace
+namespace invconv_internal {
 int sm_count()
 {
-    static std::atomic<int> cached{0};
-    int v = cached.load();
-    if (v > 0) return v;
+    static std::atomic<int> cached[64];
     int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 148; }
+    const int v = cached[dev].load();
+    if (v > 0) return v;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
         cudaGetLastError();
         return 148;            // B200; only used for planning when no device is present
     }
-    cached.store(n);
+    cached[dev].store(n);
     return n;
 }
+}  // namespace invconv_internal
+namespace {
 
 TeamPlan team_plan(int B, int C, int H, int W, int k)
 {
@@ -517,7 +521,7 @@ int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, 
         auto kern = bwd ? team_solve_kernel<true> : team_solve_kernel<false>;
         const int rc = set_smem_limit(kern, sm);
         if (rc) return rc;
-        kern<<<g.C + (g.C + 31) / 32, 512, sm, st>>>(w, A, g.C, g.k);
+        kern<<<g.C + (g.C + 31) / 32, 512, sm, st>>>(w, A, g.C, g.k, nullptr, 0, 0u);
         const int rl = check_launch();
         if (rl) return rl;
     }
@@ -548,10 +552,46 @@ int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, 
     return INVCONV_UNSUPPORTED;
 }
 
+// ---------------------------------------------------------------- tensor family
+TensorPlan tensor_plan(int B, int C, int H, int W, int k)
+{
+    if (team_solve_smem(C, k) > kMaxDynSmem) return TensorPlan{};
+    return plan_tensor(B > 0 ? B : 1, C, H, W, k, kMaxDynSmem, sm_count());
+}
+
+// Workspace: control words, transformed kernel [k*k][C][C] (+ C*C floats of slack shared with the team
+// family's layout), grad_w partial sums, then the packed tensor-core operands.
+size_t tensor_wop_offset(int B, int C, int H, int W, int k)
+{
+    const size_t na = sizeof(float) * (size_t)k * k * C * C;
+    const GradWPlan gp = gradw_plan(B, C, H, W, k);
+    const int shares = gp.nbc > gp.nbc_all ? gp.nbc : gp.nbc_all;
+    const size_t base = INVCONV_WS_CONTROL_BYTES + na + sizeof(float) * (size_t)C * C + (gp.ok ? na * shares : 0);
+    return (base + 255) & ~(size_t)255;
+}
+
+size_t tensor_workspace_bytes(int B, int C, int H, int W, int k)
+{
+    const TensorPlan pl = tensor_plan(B, C, H, W, k);
+    if (!pl.ok) return 0;
+    return tensor_wop_offset(B, C, H, W, k) + pl.wop_bytes;
+}
+
+// Plain or transposed solve on the tensor cores: kernel transform, operand packing, wavefront.
+int launch_tensor(bool bwd, const float* rhs, const float* w, float* out, Geom g, void* ws, cudaStream_t st)
+{
+    const TensorPlan pl = tensor_plan(g.B, g.C, g.H, g.W, g.k);
+    if (!pl.ok) return INVCONV_UNSUPPORTED;
+    float* A = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES);
+    unsigned char* wop = static_cast<unsigned char*>(ws) + tensor_wop_offset(g.B, g.C, g.H, g.W, g.k);
+    return invconv_internal::tensor_launch(pl, bwd, rhs, w, out, g, A, wop, st);
+}
+
 // ---------------------------------------------------------------- dispatch
 int auto_path(int B, int C, int H, int W, int k)
 {
     if (plan_warp(B > 0 ? B : 1, C, H, W, k, true).ok) return INVCONV_PATH_WARP;
+    if (tensor_plan(B, C, H, W, k).ok) return INVCONV_PATH_TENSOR;
     if (team_plan(B, C, H, W, k).ok) return INVCONV_PATH_TEAM;
     return INVCONV_PATH_GENERIC;
 }
@@ -566,6 +606,7 @@ size_t workspace_bytes_for(int path, int B, int C, int H, int W, int k)
 {
     if (path == INVCONV_PATH_WARP) return warp_workspace_bytes(B, C, H, W, k);
     if (path == INVCONV_PATH_TEAM) return team_workspace_bytes(B, C, H, W, k);
+    if (path == INVCONV_PATH_TENSOR) return tensor_workspace_bytes(B, C, H, W, k);
     return 0;
 }
 
@@ -582,6 +623,8 @@ int launch_forward(int path, const float* y, const float* w, float* x, Geom g,
         return launch_warp(false, y, w, x, nullptr, nullptr, g, ws, st);
     case INVCONV_PATH_TEAM:
         return launch_team(false, y, w, x, g, ws, st);
+    case INVCONV_PATH_TENSOR:
+        return launch_tensor(false, y, w, x, g, ws, st);
     default:
         return INVCONV_UNSUPPORTED;
     }
@@ -609,6 +652,14 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
     case INVCONV_PATH_TEAM: {
         if (g.B > 0) {
             const int rc = launch_team(true, gx, w, gy, g, ws, st);
+            if (rc) return rc;
+        }
+        if (gw) return launch_gradw(gy, x, gw, g, ws, st);
+        return INVCONV_OK;
+    }
+    case INVCONV_PATH_TENSOR: {
+        if (g.B > 0) {
+            const int rc = launch_tensor(true, gx, w, gy, g, ws, st);
             if (rc) return rc;
         }
         if (gw) return launch_gradw(gy, x, gw, g, ws, st);
@@ -892,7 +943,7 @@ int invconv_backward_noalloc(const float* grad_x, const float* x, const float* w
 
 int invconv_set_path(int path)
 {
-    if (path < INVCONV_PATH_AUTO || path > INVCONV_PATH_TEAM) return -1;
+    if (path < INVCONV_PATH_AUTO || path > INVCONV_PATH_TENSOR) return -1;
     return g_forced_path.exchange(path);
 }
 
@@ -906,13 +957,14 @@ int invconv_get_status(void* stream, int* device_status_out)
 {
     if (!device_status_out) return INVCONV_BAD_ARG;
     if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) { cudaGetLastError(); return INVCONV_CUDA_ERROR; }
-    int v = 0;
+    int v = 0, vt = 0;
     if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return INVCONV_CUDA_ERROR; }
     if (v != 0) {
         const int zero = 0;
         cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int));
     }
-    *device_status_out = v;
+    if (invconv_internal::tensor_read_clear_status(&vt) != INVCONV_OK) return INVCONV_CUDA_ERROR;
+    *device_status_out = v > vt ? v : vt;
     return INVCONV_OK;
 }
 

@@ -1,0 +1,37 @@
+// Host-side declarations shared by the translation units of the library (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+
+#include "common.cuh"
+#include "tensor_plan.h"
+
+namespace invconv_internal {
+
+constexpr size_t kMaxDynSmem = 226 * 1024;   // 227 KiB per CTA minus the kernels' static shared memory
+
+// Counts the launch and turns cudaGetLastError into a status code.
+int check_launch();
+
+// Multiprocessors of the current device (cached per device).
+int sm_count();
+
+template <typename Kern>
+inline int set_smem_limit(Kern kern, size_t smem)
+{
+    if (smem <= 48 * 1024) return INVCONV_OK;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        cudaGetLastError();
+        return INVCONV_CUDA_ERROR;
+    }
+    return INVCONV_OK;
+}
+
+// tensor_lib.cu: the tcgen05 wavefront (kernel transform into A, operand packing into wop, solve).
+int tensor_launch(const invconv::TensorPlan& pl, bool bwd, const float* rhs, const float* w, float* out,
+                  invconv::Geom g, float* A, unsigned char* wop, cudaStream_t st);
+int tensor_read_clear_status(int* status_out);
+
+}  // namespace invconv_internal

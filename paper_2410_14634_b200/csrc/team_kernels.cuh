@@ -24,6 +24,7 @@
 #pragma once
 
 #include <cooperative_groups.h>
+#include <cuda_bf16.h>
 #include <cstdio>
 #include <cstdlib>
 #include <type_traits>
@@ -50,7 +51,8 @@ namespace cg = cooperative_groups;
 // separate array so that no thread reads a row another thread is rewriting.
 // ---------------------------------------------------------------------------
 template <bool BWD>
-__global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K)
+__global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K,
+                                                         unsigned char* __restrict__ wop, int NCH, unsigned wbytes)
 {
     extern __shared__ __align__(128) float sm[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the wavefront kernel may set itself up meanwhile
@@ -142,11 +144,31 @@ __global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict
         }
         __syncthreads();
     }
+    if (wop == nullptr) {
+        for (int e = tid; e < C * NC; e += NT) {
+            const int col = e / C, a = e - col * C;               // a fastest: coalesced stores
+            const float v = Y[a * NC + col];
+            if (ident) A[(size_t)(c0 + col) * C + a] = v;         // A[0][b' = c0 + col][a]
+            else if (col != ctr) A[((size_t)(KK - 1 - col) * C + b) * C + a] = v;
+        }
+        return;
+    }
+    // Tensor-core operand form instead (see tensor_kernels.cuh): per CTA rank r = chunk / NCH one block
+    //   [dh][chunk % NCH][plane 0,1: tf32 hi | plane 2: bf16 remainder | plane 3: bf16 value][row = dw*C + a][16 bytes],
+    // chunk = input channel / 8; the sign is flipped for every tap but tap 0.
+    const int KC = K * C;
     for (int e = tid; e < C * NC; e += NT) {
-        const int col = e / C, a = e - col * C;               // a fastest: coalesced stores
-        const float v = Y[a * NC + col];
-        if (ident) A[(size_t)(c0 + col) * C + a] = v;         // A[0][b' = c0 + col][a]
-        else if (col != ctr) A[((size_t)(KK - 1 - col) * C + b) * C + a] = v;
+        const int col = e / C, a = e - col * C;
+        if (!ident && col == ctr) continue;
+        const int tap = ident ? 0 : KK - 1 - col, ci = ident ? c0 + col : b;
+        const float v = ident ? Y[a * NC + col] : -Y[a * NC + col];
+        const float hi = tf32_hi(v);
+        const int chunk = ci >> 3, j = ci & 7, r = chunk / NCH, cl = chunk - r * NCH;
+        const int dh = tap / K, dw = tap - dh * K, row = dw * C + a;
+        unsigned char* blk = wop + (size_t)r * wbytes + (size_t)((dh * NCH + cl) * 4) * KC * 16;
+        *reinterpret_cast<float*>(blk + ((size_t)(j >> 2) * KC + row) * 16 + (j & 3) * 4) = hi;
+        *reinterpret_cast<__nv_bfloat16*>(blk + ((size_t)2 * KC + row) * 16 + j * 2) = __float2bfloat16_rn(v - hi);
+        *reinterpret_cast<__nv_bfloat16*>(blk + ((size_t)3 * KC + row) * 16 + j * 2) = __float2bfloat16_rn(v);
     }
 }
 

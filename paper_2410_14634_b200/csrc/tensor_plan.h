@@ -1,0 +1,61 @@
+// Launch geometry of the tensor-core wavefront (host side; see tensor_kernels.cuh for the kernel).
+#pragma once
+
+#include <stddef.h>
+
+namespace invconv {
+
+struct TensorPlan {
+    bool ok = false;
+    int R = 0;          // CTAs per cluster = C / (8 * NCH)
+    int NCH = 0;        // 8-channel chunks of the contraction per CTA
+    int I = 0;          // images per group (128 lanes / HP)
+    int HP = 0;         // image rows padded to 8 or 16
+    int S = 0;          // accumulator slots
+    int ngroups = 0, ncl = 0;
+    unsigned tmem_cols = 0;
+    unsigned wbytes = 0;            // packed kernel bytes per CTA
+    unsigned off_stage = 0, off_x = 0, off_y = 0, off_recv = 0, off_bar = 0;
+    unsigned stage_img = 0;         // floats between the images of the staged slice
+    size_t smem = 0;
+    size_t wop_bytes = 0;           // packed kernel, all CTAs
+};
+
+constexpr int kTensorThreads = 416;     // warps 0-7: accumulators -> solved pixels; warp 8: MMA issue; warps 9-12: right-hand side
+
+inline TensorPlan plan_tensor(int B, int C, int H, int W, int K, size_t max_smem, int sms)
+{
+    TensorPlan pl;
+    if (K < 2 || K > 5 || H > 16 || C % 16 != 0 || C > 64 || (H * W) % 4 != 0 || B < 1) return pl;
+    pl.NCH = 1;
+    pl.R = C / 8;
+    if (pl.R < 2 || pl.R > 8) return pl;
+    pl.HP = H <= 8 ? 8 : 16;
+    pl.I = 128 / pl.HP;
+    pl.S = 2 * (K - 1);
+    if (pl.S * C > 512) return pl;
+    unsigned cols = 32;
+    while (cols < (unsigned)(pl.S * C)) cols *= 2;
+    pl.tmem_cols = cols;
+    const int CS = 8 * pl.NCH, KC = K * C, ROWS = (K - 1) * pl.I + 128;
+    auto up = [](size_t v) { return (v + 127) & ~(size_t)127; };
+    pl.wbytes = (unsigned)(K * pl.NCH * KC * 64);
+    pl.stage_img = (unsigned)(CS * H * W + 4);
+    size_t off = up(pl.wbytes);
+    pl.off_stage = (unsigned)off;  off = up(off + sizeof(float) * (size_t)pl.I * pl.stage_img);
+    pl.off_x = (unsigned)off;      off = up(off + 2 * (size_t)pl.NCH * 4 * ROWS * 16);
+    pl.off_y = (unsigned)off;      off = up(off + 2 * (size_t)pl.NCH * 4 * 128 * 16);
+    pl.off_recv = (unsigned)off;   off = up(off + 2 * (size_t)(pl.R - 1) * 128 * CS * sizeof(float));
+    pl.off_bar = (unsigned)off;    off += 256;
+    pl.smem = off;
+    if (pl.smem > max_smem) return pl;
+    pl.ngroups = (B + pl.I - 1) / pl.I;
+    int ncl = sms / pl.R;
+    if (ncl < 1) return pl;
+    pl.ncl = pl.ngroups < ncl ? pl.ngroups : ncl;
+    pl.wop_bytes = (size_t)pl.R * pl.wbytes;
+    pl.ok = true;
+    return pl;
+}
+
+}  // namespace invconv

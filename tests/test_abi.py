@@ -69,9 +69,9 @@ def test_dispatch_and_workspace_planning_need_no_device(library):
     library.invconv_workspace_bytes.restype = ctypes.c_size_t
     library.invconv_workspace_bytes.argtypes = [ctypes.c_int] * 5
     library.invconv_path_for.argtypes = [ctypes.c_int] * 5
-    GENERIC, WARP, TEAM = 1, 2, 3
+    GENERIC, WARP, TEAM, TENSOR = 1, 2, 3, 4
     want = {"pr1": WARP, "mnist": WARP, "cifar": WARP, "large64": WARP, "large256": WARP,
-            "cifar_sq": TEAM, "wide48_k3": TEAM, "wide48_k5": TEAM, "wide96_k3": TEAM, "wide96_k5": TEAM}
+            "cifar_sq": TEAM, "wide48_k3": TENSOR, "wide48_k5": TENSOR, "wide96_k3": TEAM, "wide96_k5": TEAM}
     for s in workloads.SHAPES:
         assert library.invconv_path_for(s.B, s.C, s.H, s.W, s.k) == want[s.name], s.name
         need = library.invconv_workspace_bytes(s.B, s.C, s.H, s.W, s.k)

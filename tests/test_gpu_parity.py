@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 TOL_X = 1e-4
 TOL_GW = 1e-3
 
-PATHS = {"auto": 0, "generic": 1, "warp": 2, "team": 3}
+PATHS = {"auto": 0, "generic": 1, "warp": 2, "team": 3, "tensor": 4}
 
 
 @pytest.fixture(scope="module")
@@ -38,11 +38,14 @@ def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def run_or_skip(binding, fn, *args, **kw):
+def run_or_skip(binding, path, fn, *args, **kw):
+    """A forced family may decline a shape (skip); the automatic choice must serve every shape."""
     try:
         return fn(*args, **kw)
     except binding.InvConvError as e:
         if e.status == binding.UNSUPPORTED:
+            if path == "auto":
+                pytest.fail("the automatic dispatch returned UNSUPPORTED")
             pytest.skip("this kernel family does not serve the shape")
         raise
 
@@ -55,8 +58,8 @@ def check_all(binding, oracle, w, y, gx, path, tol_x=TOL_X, tol_gw=TOL_GW):
     binding.invconv_set_path(PATHS[path])
     try:
         wd, yd, gxd = dev(w), dev(y), dev(gx)
-        x = run_or_skip(binding, binding.invconv_forward, yd, wd)
-        gy, gw = run_or_skip(binding, binding.invconv_backward, gxd, x, wd)
+        x = run_or_skip(binding, path, binding.invconv_forward, yd, wd)
+        gy, gw = run_or_skip(binding, path, binding.invconv_backward, gxd, x, wd)
         x_ref = oracle.invconv_forward(y, w)
         gy_ref, gw_ref = oracle.invconv_backward(gx, x_ref, w)
         # backward again from the oracle's x rounded to fp32 (separates forward from backward error)
@@ -82,7 +85,7 @@ def check_all(binding, oracle, w, y, gx, path, tol_x=TOL_X, tol_gw=TOL_GW):
 
 # ------------------------------------------------------------------ the ten benchmark shapes, full size
 
-@pytest.mark.parametrize("path", ["auto", "generic", "warp", "team"])
+@pytest.mark.parametrize("path", ["auto", "generic", "warp", "team", "tensor"])
 @pytest.mark.parametrize("name", [s.name for s in workloads.SHAPES])
 def test_benchmark_shapes_full_size(B, oracle, name, path):
     s, w, y, gx = workloads.make(name)
@@ -101,10 +104,15 @@ EDGE = [  # (B, C, H, W, k)
     (1, 2, 16, 16, 11), (1, 1, 65, 66, 3), (1, 3, 100, 20, 3), (5, 1, 28, 28, 3),
     (1, 3, 100, 200, 3), (2, 1, 250, 260, 5), (1, 2, 70, 500, 2),       # larger than shared memory: global-memory mode
     (1, 1, 250, 257, 3), (1, 2, 130, 301, 5), (1, 4, 96, 180, 2), (1, 3, 200, 160, 3),   # ... ragged widths (4-byte ring copies), ring too large
+    (1, 2, 12, 12, 9), (2, 3, 20, 24, 9),                                 # the paper's ablation also runs k = 9
+    # tensor-core family: every channel count it serves, k = 2..5, fewer rows than lanes, wide and narrow images,
+    # batches that do not fill a group of images, several groups per cluster
+    (9, 16, 16, 16, 3), (3, 32, 8, 8, 5), (17, 48, 16, 4, 2), (5, 64, 12, 16, 4), (1, 48, 16, 16, 5),
+    (20, 16, 7, 12, 5), (2, 32, 16, 32, 3), (200, 16, 4, 4, 3), (33, 48, 2, 2, 3), (4, 64, 16, 16, 5),
 ]
 
 
-@pytest.mark.parametrize("path", ["auto", "generic", "warp", "team"])
+@pytest.mark.parametrize("path", ["auto", "generic", "warp", "team", "tensor"])
 @pytest.mark.parametrize("shape", EDGE, ids=lambda s: "x".join(map(str, s)))
 def test_edge_shapes(B, oracle, shape, path):
     Bn, C, H, W, k = shape
@@ -238,7 +246,7 @@ def test_grad_w_many_channels_fma_and_tensor_pipe(B, oracle, shape, mma, monkeyp
     gy_ref, gw_ref = oracle.invconv_backward(gx, x_ref, w)
     B.invconv_set_path(PATHS["team"])
     try:
-        _, gw = run_or_skip(B, B.invconv_backward, dev(gx), dev(x_ref.astype(np.float32)), dev(w))
+        _, gw = run_or_skip(B, "forced", B.invconv_backward, dev(gx), dev(x_ref.astype(np.float32)), dev(w))
     finally:
         B.invconv_set_path(0)
     err = nmax_err(gw.cpu().numpy(), gw_ref)
