@@ -194,6 +194,11 @@ int invconv_set_path(int path);
 /* The family AUTO would pick for this shape (an invconv_path value). */
 int invconv_path_for(int B, int C, int H, int W, int k);
 
+/* CTAs per thread-block cluster of the wavefront kernel AUTO would launch for this shape (1 = no cluster):
+ * more than one means that neighbouring diagonals are exchanged through distributed shared memory, which is
+ * what sets the latency of one dependent step (Section 3.3: H+W-1 sequential steps). */
+int invconv_cluster_size_for(int B, int C, int H, int W, int k);
+
 /* Synchronises `stream`, then reports and clears the device-side status word
  * of the current device: INVCONV_OK, or INVCONV_TIMEOUT if a bounded wait
  * inside a kernel gave up since the last query (its outputs are then invalid).

@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.invconv_step_host.argtypes = [vp] * 7 + [ci] * 5 + [vp, sz, vp]
         L.invconv_set_path.argtypes = [ci]
         L.invconv_path_for.argtypes = [ci] * 5
+        L.invconv_cluster_size_for.argtypes = [ci] * 5
+        L.invconv_cluster_size_for.restype = ci
         L.invconv_get_status.argtypes = [vp, ctypes.POINTER(ci)]
         L.invconv_probe_step_latency.argtypes = [ci, ci, vp, vp]
         L.invconv_status_string.argtypes = [ci]
@@ -268,6 +270,10 @@ def invconv_set_path(path: int) -> int:
 
 def invconv_path_for(B: int, C: int, H: int, W: int, k: int) -> int:
     return int(lib().invconv_path_for(B, C, H, W, k))
+
+
+def invconv_cluster_size_for(B: int, C: int, H: int, W: int, k: int) -> int:
+    return int(lib().invconv_cluster_size_for(B, C, H, W, k))
 
 
 def invconv_get_status(stream: Optional[torch.cuda.Stream] = None, device="cuda:0") -> int:

@@ -953,6 +953,16 @@ int invconv_path_for(int B, int C, int H, int W, int k)
     return auto_path(B, C, H, W, k);
 }
 
+int invconv_cluster_size_for(int B, int C, int H, int W, int k)
+{
+    if (check_shape(B, C, H, W, k) != INVCONV_OK) return -1;
+    switch (auto_path(B, C, H, W, k)) {
+    case INVCONV_PATH_TENSOR: return tensor_plan(B, C, H, W, k).R;
+    case INVCONV_PATH_TEAM: return team_plan(B, C, H, W, k).R;
+    default: return 1;
+    }
+}
+
 int invconv_get_status(void* stream, int* device_status_out)
 {
     if (!device_status_out) return INVCONV_BAD_ARG;
