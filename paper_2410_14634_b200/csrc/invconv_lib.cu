@@ -570,11 +570,42 @@ size_t tensor_wop_offset(int B, int C, int H, int W, int k)
     return (base + 255) & ~(size_t)255;
 }
 
+GradWTensorPlan gradw_tensor_plan(int B, int C, int H, int W, int k)
+{
+    return plan_gradw_tensor(B > 0 ? B : 1, C, H, W, k, kMaxDynSmem, sm_count());
+}
+
+size_t tensor_gradw_offset(int B, int C, int H, int W, int k)
+{
+    return (tensor_wop_offset(B, C, H, W, k) + tensor_plan(B, C, H, W, k).wop_bytes + 255) & ~(size_t)255;
+}
+
 size_t tensor_workspace_bytes(int B, int C, int H, int W, int k)
 {
     const TensorPlan pl = tensor_plan(B, C, H, W, k);
     if (!pl.ok) return 0;
-    return tensor_wop_offset(B, C, H, W, k) + pl.wop_bytes;
+    const GradWTensorPlan gt = gradw_tensor_plan(B, C, H, W, k);
+    const size_t na = sizeof(float) * (size_t)k * k * C * C;
+    return tensor_gradw_offset(B, C, H, W, k) + (gt.ok ? na * gt.S : 0);
+}
+
+// grad_w through the tensor-core correlation kernel and the fixed-order reduction over its shares.
+int launch_gradw_tensor(const float* gy, const float* x, float* gw, Geom g, void* ws, cudaStream_t st)
+{
+    const GradWTensorPlan gt = gradw_tensor_plan(g.B, g.C, g.H, g.W, g.k);
+    const bool aligned = ((reinterpret_cast<uintptr_t>(gy) | reinterpret_cast<uintptr_t>(x)) & 15) == 0;
+    if (!gt.ok || !aligned || g.B == 0) return launch_gradw(gy, x, gw, g, ws, st);
+    float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + tensor_gradw_offset(g.B, g.C, g.H, g.W, g.k));
+    const int rc = invconv_internal::gradw_tensor_launch(gt, gy, x, partials, g, st);
+    if (rc) return rc;
+    const size_t na = (size_t)g.k * g.k * g.C * g.C;
+    if (na < 16384) {
+        gradw_reduce_kernel<4><<<(int)((na + 63) / 64), 256, 0, st>>>(partials, gw, gt.S, g.C, g.k);
+    } else {
+        const int blocks = (int)((na + 255) / 256 < 4096 ? (na + 255) / 256 : 4096);
+        gradw_reduce_kernel<1><<<blocks, 256, 0, st>>>(partials, gw, gt.S, g.C, g.k);
+    }
+    return check_launch();
 }
 
 // Plain or transposed solve on the tensor cores: kernel transform, operand packing, wavefront.
@@ -662,7 +693,7 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
             const int rc = launch_tensor(true, gx, w, gy, g, ws, st);
             if (rc) return rc;
         }
-        if (gw) return launch_gradw(gy, x, gw, g, ws, st);
+        if (gw) return launch_gradw_tensor(gy, x, gw, g, ws, st);
         return INVCONV_OK;
     }
     default:

@@ -34,4 +34,8 @@ int tensor_launch(const invconv::TensorPlan& pl, bool bwd, const float* rhs, con
                   invconv::Geom g, float* A, unsigned char* wop, cudaStream_t st);
 int tensor_read_clear_status(int* status_out);
 
+// tensor_lib.cu: the tcgen05 correlation kernel of grad_w; partial sums [pl.S][k*k][C][C] go to `partials`.
+int gradw_tensor_launch(const invconv::GradWTensorPlan& pl, const float* gy, const float* x, float* partials,
+                        invconv::Geom g, cudaStream_t st);
+
 }  // namespace invconv_internal

@@ -10,6 +10,7 @@
 #include "lib_internal.h"
 #include "team_kernels.cuh"      // team_solve_kernel: the kernel transform L^-1 W_delta
 #include "tensor_kernels.cuh"
+#include "gradw_tensor.cuh"
 
 using namespace invconv;
 
@@ -73,6 +74,34 @@ int tensor_launch(const TensorPlan& pl, bool bwd, const float* rhs, const float*
     X(3, 2) X(3, 3) X(3, 4) X(3, 5) X(4, 2) X(4, 3) X(4, 4) X(4, 5)
 #undef X
     return INVCONV_UNSUPPORTED;
+}
+
+int gradw_tensor_launch(const GradWTensorPlan& pl, const float* gy, const float* x, float* partials, Geom g, cudaStream_t st)
+{
+    auto kern = gradw_tensor_kernel;
+    const int rc = set_smem_limit(kern, pl.smem);
+    if (rc) return rc;
+    GradWTensorParams prm;
+    prm.gy = gy; prm.x = x; prm.partials = partials;
+    prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W; prm.K = g.k;
+    prm.RB = pl.RB; prm.Wp = pl.Wp; prm.nbands = pl.nbands; prm.S = pl.S; prm.nk = pl.nk;
+    prm.tmem_cols = pl.tmem_cols; prm.planeA = pl.planeA; prm.planeB = pl.planeB; prm.stage_bytes = pl.stage_bytes;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(pl.grid);
+    cfg.blockDim = dim3(kGradWTensorProducers + 32 * g.k);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // set-up overlaps the tail of the solve
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
+    if (e != cudaSuccess) {
+        std::fprintf(stderr, "invconv: grad_w tensor launch failed: %s\n", cudaGetErrorString(e));
+        cudaGetLastError();
+        return INVCONV_CUDA_ERROR;
+    }
+    return check_launch();
 }
 
 int tensor_read_clear_status(int* status_out)

@@ -58,4 +58,41 @@ inline TensorPlan plan_tensor(int B, int C, int H, int W, int K, size_t max_smem
     return pl;
 }
 
+struct GradWTensorPlan {
+    bool ok = false;
+    int RB = 0, Wp = 0, nbands = 0, S = 0, grid = 0, nk = 0;
+    unsigned tmem_cols = 0, planeA = 0, planeB = 0, stage_bytes = 0;
+    size_t smem = 0;
+};
+
+constexpr int kGradWTensorProducers = 256;    // warps 0-7 stage the operands (0-3 also write the result); warps 8.. issue the MMAs, one per kernel column
+
+inline GradWTensorPlan plan_gradw_tensor(int B, int C, int H, int W, int K, size_t max_smem, int sms)
+{
+    GradWTensorPlan pl;
+    if (C % 16 != 0 || C < 16 || C > 128 || K * C > 512 || B < 1 || K > 5 || W % 4 != 0) return pl;
+    pl.Wp = W;
+    for (pl.RB = H >= 4 ? 4 : 2; pl.RB >= 2; pl.RB -= 2) {
+        // one stage: grad_y and K shifted copies of x, [quad][channel][4 pixels] each, plus room for the rows
+        // C..127 that the MMA reads (and ignores) behind the last quad plane
+        pl.stage_bytes = (unsigned)(((size_t)(K + 1) * (pl.RB * W / 4) * (C + 1) * 16 + 128 * 16 + 127) & ~(size_t)127);
+        pl.smem = 2 * (size_t)pl.stage_bytes + 256;
+        if (pl.smem <= max_smem) break;
+    }
+    if (pl.RB < 2 || (pl.RB * W) % 8 != 0 || C * pl.RB * (W / 4) > 8 * kGradWTensorProducers) return pl;
+    pl.nbands = (H + pl.RB - 1) / pl.RB;
+    pl.nk = pl.RB * W / 8;
+    pl.planeA = pl.planeB = (unsigned)(C + 1) * 16;
+    pl.S = sms / K;
+    if (pl.S < 1) return pl;
+    const int units = B * pl.nbands;
+    if (pl.S > units) pl.S = units;
+    pl.grid = pl.S * K;
+    unsigned cols = 32;
+    while (cols < (unsigned)(K * C)) cols *= 2;
+    pl.tmem_cols = cols;
+    pl.ok = true;
+    return pl;
+}
+
 }  // namespace invconv
