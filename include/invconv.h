@@ -79,7 +79,12 @@ int invconv_forward(const float* y, const float* w, float* x,
  *                                   summed over the batch; 0 outside the mask.
  *   grad_x [B,C,H,W] in, x [B,C,H,W] in (the saved forward output), w in,
  *   grad_y [B,C,H,W] out, grad_w [C,C,k,k] out.  grad_w may be NULL (skip it);
- *   grad_y must be non-NULL (grad_w is computed from it). */
+ *   grad_y must be non-NULL (grad_w is computed from it).
+ * Precision: the solves accumulate in fp32 throughout (the tensor-core family splits every operand into a
+ * tf32 part and a bf16 remainder, so its products carry about 19 bits).  For C >= 12 the sum over pixels of
+ * grad_w runs on the tensor pipe with its two operands rounded to tf32 (10-bit mantissa) and fp32
+ * accumulation: each entry is then accurate to about 3e-4 of the LARGEST entry of grad_w, not of itself;
+ * INVCONV_OPT_GRADW_TENSOR_PIPE = 0 selects the fp32 kernel instead. */
 int invconv_backward(const float* grad_x, const float* x, const float* w,
                      float* grad_y, float* grad_w,
                      int B, int C, int H, int W, int k, void* stream);
@@ -173,9 +178,13 @@ int invconv_step_host(const float* y_host, const float* w_host, const float* gra
  *    warp-shuffle kernel family only.  Shapes that family does not serve return
  *    INVCONV_UNSUPPORTED; shapes whose scratch would exceed the fixed array
  *    return INVCONV_WORKSPACE_TOO_SMALL.  Nothing is launched in either case.
- *  - Calls cudaMalloc, cudaFree or any other allocating routine never.
- *  - The first call on each device looks up the array's device address (with
- *    that device current) and caches it; make that first call before any
+ *  - The library itself calls neither cudaMalloc nor cudaFree nor any other
+ *    allocating routine here.  The CUDA runtime, however, loads a kernel's code
+ *    the first time that kernel is launched, and that may allocate: call once
+ *    per (shape, grad_w NULL or not) on each device during start-up, before
+ *    memory is frozen.
+ *  - The first call on each device also looks up the array's device address
+ *    (with that device current) and caches it; make that first call before any
  *    stream capture begins on the device.
  *  - All calls on a device share the one array.  Each call clears the control
  *    words it relies on, on `stream`, before its kernel runs, so a call may
@@ -209,17 +218,33 @@ int invconv_get_status(void* stream, int* device_status_out);
  * for a communication mechanism, with no other work on the chain:
  *   mechanism 0: warp shuffle + one FMA (lane = image row);
  *   mechanism 1: shared-memory store, block barrier, load, one FMA;
- *   mechanism 2: store to a cluster peer's shared memory, cluster barrier, load, one FMA;
- *   mechanism 3: one dependent FMA (the latency of a single accumulator);
- *   mechanism 4: two broadcast 16-byte shared-memory loads feeding 24 FMAs on six accumulators
- *                (one "group" of the wide-channel kernels' inner loop, 8 warps resident);
- *   mechanism 5: the arithmetic of one wavefront step for three channels and a 3x3 kernel held in
- *                registers (six shuffles, 81 FMAs, window rotation; no shared memory).
+ *   mechanism 2: store to a cluster peer's shared memory, cluster barrier, load, one FMA.
  * Runs a chain of `steps` dependent steps in one CTA (cluster of 2 for 2) and
  * writes the elapsed SM clock cycles to cycles_out[0] and the chain's final
  * value to cycles_out[1] (device pointer to two 64-bit words).  Used for the
  * critical-path bound of 2*(H+W-1) dependent steps (Section 3.3, complexity). */
 int invconv_probe_step_latency(int mechanism, int steps, unsigned long long* cycles_out, void* stream);
+
+/* Self-test of the bounded device-side waits: launches one small kernel that waits, with a limit of
+ * `limit_cycles` SM clock cycles (1 <= limit_cycles <= 2^24), on a barrier that nothing completes.  The wait
+ * runs out, the kernel raises the device status word to INVCONV_TIMEOUT and returns normally; the context
+ * stays usable.  invconv_get_status then reports INVCONV_TIMEOUT once. */
+int invconv_selftest_wait_timeout(unsigned limit_cycles, void* stream);
+
+/* Development and test controls -- not needed in normal use.  They force one of two equivalent kernels or
+ * launch modes so that tests and measurements can compare them; results are the same within rounding.
+ * invconv_set_option returns the previous value, or -1 for an unknown option.  Process-wide. */
+enum invconv_option {
+    INVCONV_OPT_WARP_RING = 0,       /* 1 (default): images larger than shared memory stream through a ring; 0: global-memory mode */
+    INVCONV_OPT_WARP_CHANNEL_SPLIT,  /* 1 (default): lane = (row, channel) walk for C >= 3, k = 5; 0: one lane per row */
+    INVCONV_OPT_GRADW_SEPARATE,      /* -1 (default): by shape; 0: grad_w inside the warp wavefront; 1: separate pixel-parallel kernel */
+    INVCONV_OPT_GRADW_TENSOR_PIPE,   /* 1 (default): many-channel grad_w on the tensor pipe (tf32 operands); 0: fp32 FMA kernel */
+    INVCONV_OPT_TEAM_VARIANT,        /* 0 (default): by shape; 1: channel-slice kernel; 2: pixel-team kernel */
+    INVCONV_OPT_TEAM_CLUSTER,        /* 0 (default): by shape; 1..8: force the cluster size of the channel-slice kernel */
+    INVCONV_OPT_DEPENDENT_LAUNCH,    /* 1 (default): programmatic dependent launch between the library's kernels; 0: off */
+    INVCONV_OPT_COUNT
+};
+int invconv_set_option(int option, int value);
 
 /* Number of kernels this library has launched (or captured into a CUDA graph)
  * from this process since it was loaded. */

@@ -56,6 +56,10 @@ def lib() -> ctypes.CDLL:
         L.invconv_step_scratch_bytes.restype = sz
         L.invconv_step_host.argtypes = [vp] * 7 + [ci] * 5 + [vp, sz, vp]
         L.invconv_set_path.argtypes = [ci]
+        L.invconv_set_option.argtypes = [ci, ci]
+        L.invconv_set_option.restype = ci
+        L.invconv_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp]
+        L.invconv_selftest_wait_timeout.restype = ci
         L.invconv_path_for.argtypes = [ci] * 5
         L.invconv_cluster_size_for.argtypes = [ci] * 5
         L.invconv_cluster_size_for.restype = ci
@@ -262,6 +266,27 @@ class HostStep:
                                            self.logdet.data_ptr(), B, C, H, W, k, self.scratch.data_ptr(),
                                            self.scratch.numel(), _stream_ptr(stream, self.device)),
                    "invconv_step_host")
+
+
+# invconv_option values (development and test controls, see include/invconv.h)
+(OPT_WARP_RING, OPT_WARP_CHANNEL_SPLIT, OPT_GRADW_SEPARATE, OPT_GRADW_TENSOR_PIPE, OPT_TEAM_VARIANT,
+ OPT_TEAM_CLUSTER, OPT_DEPENDENT_LAUNCH) = range(7)
+
+
+def invconv_set_option(option: int, value: int) -> int:
+    """Set a development/test control; returns the previous value."""
+    prev = int(lib().invconv_set_option(option, value))
+    if prev == -1 and not (0 <= option < 7):
+        raise ValueError("unknown option")
+    return prev
+
+
+def invconv_selftest_wait_timeout(limit_cycles: int = 20000, stream: Optional[torch.cuda.Stream] = None,
+                                  device="cuda:0") -> None:
+    """Launch the kernel whose bounded wait runs out on purpose (see include/invconv.h)."""
+    with torch.cuda.device(device):
+        _check(lib().invconv_selftest_wait_timeout(limit_cycles, _stream_ptr(stream, device)),
+               "invconv_selftest_wait_timeout")
 
 
 def invconv_set_path(path: int) -> int:

@@ -189,9 +189,6 @@ __global__ void __launch_bounds__(32 * (ALLDH ? K * K : TC * K)) gradw_mma_kerne
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
-#ifdef INVCONV_GW_TIMING
-    long long tm_[5]; tm_[0] = clock64(); tm_[1] = tm_[2] = tm_[0];
-#endif
     // channels beyond C (padding of the last tile) stay zero; the others are overwritten by every image
     for (int c = nco + warp; c < TB; c += nwarps)
         for (int i = lane; i < p.plane; i += 32) gys[c * p.plane + i] = 0.f;
@@ -214,9 +211,6 @@ __global__ void __launch_bounds__(32 * (ALLDH ? K * K : TC * K)) gradw_mma_kerne
         cp_async_commit();
         cp_async_wait<0>();
         __syncthreads();
-#ifdef INVCONV_GW_TIMING
-        tm_[1] = clock64();
-#endif
 
         const float* ga = gys + (mt * 16 + g) * p.plane + t;          // A: rows g and g + 8, pixel columns t and t + 4
         const float* xb = xs + g * p.plane + t - dw;                  // B: channel g of a group, pixels t and t + 4, shifted
@@ -238,9 +232,6 @@ __global__ void __launch_bounds__(32 * (ALLDH ? K * K : TC * K)) gradw_mma_kerne
                 }
             }
         }
-#ifdef INVCONV_GW_TIMING
-        tm_[2] = clock64();
-#endif
         __syncthreads();       // everyone is done with this image before its planes are overwritten
     }
 
@@ -252,11 +243,6 @@ __global__ void __launch_bounds__(32 * (ALLDH ? K * K : TC * K)) gradw_mma_kerne
             const int co = co0 + mt * 16 + g + (j >> 1) * 8, ci = ci0 + nt * 8 + 2 * t + (j & 1);
             if (co < C && ci < C) dst[(size_t)co * C + ci] = acc[nt][j];
         }
-#ifdef INVCONV_GW_TIMING
-    tm_[3] = clock64();
-    if (tid == 0 && blockIdx.x == 0)
-        printf("gradw_mma (cycles) block 0: staged %lld | computed %lld | written %lld\n", tm_[1] - tm_[0], tm_[2] - tm_[0], tm_[3] - tm_[0]);
-#endif
 }
 
 // grad_w[co][ci][K-1-dh][K-1-dw] = -(sum over shares), zero outside the channel mask of the centre tap.
@@ -413,14 +399,7 @@ __global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(
     // shared-memory set-up needs nothing from the predecessor kernel
     if (tid == 0) { mbar_init(&bar, 1); fence_mbar_init(); }
     asm volatile("griddepcontrol.wait;" ::: "memory");
-#ifdef INVCONV_GW_TIMING
-    long long tg_[8]; tg_[0] = clock64(); tg_[1] = tg_[2] = tg_[5] = tg_[6] = tg_[7] = tg_[0];
-#define GW_TT(i) tg_[i] = clock64()
-#else
-#define GW_TT(i) do { } while (0)
-#endif
     __syncthreads();
-    GW_TT(4);
 
     unsigned phase = 0;
     const int items = p.B * p.nbands;
@@ -446,7 +425,6 @@ __global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(
                 }
             }
             fence_proxy_async();
-            GW_TT(5);
             if (warp == 0) {
                 if (lane == 0) mbar_expect_tx(&bar, (unsigned)(C * (gv + xv) * W * 4));
                 __syncwarp();
@@ -454,9 +432,7 @@ __global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(
                 else if (lane < 2 * C)
                     bulk_g2s(xsm + ((lane - C) * XR + xskip) * xst, xsrc + (lane - C) * HW + xlo * W, (unsigned)(xv * W * 4), &bar);
             }
-            GW_TT(6);
             const bool ok = mbar_wait_bounded(&bar, phase);
-            GW_TT(7);
             phase ^= 1u;
             if (!__syncthreads_and(ok)) { if (tid == 0) raise_status(INVCONV_TIMEOUT); break; }
         } else {
@@ -485,7 +461,6 @@ __global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(
             }
             __syncthreads();
         }
-        GW_TT(1);
         const float* gq = gsm + co * RB * gst;
         const float* xq = xsm + ci * XR * xst;
         for (int q = slice; q < nq; q += NSL) {
@@ -506,7 +481,6 @@ __global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(
             }
         }
     }
-    GW_TT(2);
     // let the next kernel on the stream be scheduled only now: its CTAs would otherwise sit on the SMs (and
     // hold their registers and shared memory) for this kernel's whole run, which measured slower
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -532,12 +506,6 @@ __global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(
     __syncthreads();
     if (tid == 0) ticket = atomicAdd(p.counter, 1u);
     __syncthreads();
-    GW_TT(3);
-#ifdef INVCONV_GW_TIMING
-    if (tid == 0 && blockIdx.x == 0)
-        printf("gradw_small (cycles) block 0: first barrier %lld | zero-fill end %lld | issued %lld | arrived %lld | last load %lld (from start) | compute end %lld | partial+ticket end %lld | ticket %u of %u\n",
-               tg_[4] - tg_[0], tg_[5] - tg_[0], tg_[6] - tg_[0], tg_[7] - tg_[0], tg_[1] - tg_[0], tg_[2] - tg_[0], tg_[3] - tg_[0], ticket, gridDim.x);
-#endif
     if (ticket != gridDim.x - 1) return;
 
     // last CTA: add the CTAs' sums in CTA order, staged through shared memory sixteen bytes at a time
@@ -572,10 +540,6 @@ __global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(
         p.grad_w[((co_ * C + ci_) * K + (K - 1 - dh_)) * K + (K - 1 - dw_)] = (tap == 0 && ci_ > co_) ? 0.f : -red[e];
     }
     if (tid == 0) *p.counter = 0u;
-#ifdef INVCONV_GW_TIMING
-    GW_TT(4);
-    if (tid == 0) printf("gradw_small last CTA %d: total %lld | final reduce %lld\n", (int)blockIdx.x, tg_[4] - tg_[0], tg_[4] - tg_[3]);
-#endif
 }
 
 struct GradWSmallPlan {

@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
         const long long t0 = clock64();
         while (!mbar_try_wait(bar, parity)) {
             if (*gave_up) return;
-            if (clock64() - t0 > (1ll << 27)) { *gave_up = 1; raise_status(INVCONV_TIMEOUT); return; }
+            if (clock64() - t0 > (1ll << 24)) { *gave_up = 1; raise_status(INVCONV_TIMEOUT); return; }
         }
     };
 

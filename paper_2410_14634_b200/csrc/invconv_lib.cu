@@ -29,7 +29,9 @@ namespace {
 
 std::atomic<int> g_forced_path{INVCONV_PATH_AUTO};
 std::atomic<unsigned long long> g_kernel_launches{0};
-std::atomic<bool> g_use_pdl{std::getenv("INVCONV_NO_PDL") == nullptr};   // measurement knob: INVCONV_NO_PDL=1 disables it
+// development and test controls (invconv_set_option); defaults as documented in the header
+std::atomic<int> g_opt[INVCONV_OPT_COUNT] = {{1}, {1}, {-1}, {1}, {0}, {0}, {1}};
+inline int opt(int o) { return g_opt[o].load(std::memory_order_relaxed); }
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
@@ -129,10 +131,10 @@ template <int C, int K, bool BWD>
 int launch_warp_ck(const WarpPlan& pl, WarpParams prm, cudaStream_t st)
 {
     // global-memory mode: streamed through a shared-memory ring unless grad_w rides along in the wavefront
-    const bool ring = pl.glb && pl.ring && prm.grad_w == nullptr && std::getenv("INVCONV_NO_RING") == nullptr;
+    const bool ring = pl.glb && pl.ring && prm.grad_w == nullptr && opt(INVCONV_OPT_WARP_RING) != 0;
     // channel-split walk (its own row-block geometry) unless grad_w rides along in the wavefront
     bool cs = false;
-    if constexpr (C >= 3 && K == 5) cs = pl.cs && prm.grad_w == nullptr && std::getenv("INVCONV_NO_CS") == nullptr;
+    if constexpr (C >= 3 && K == 5) cs = pl.cs && prm.grad_w == nullptr && opt(INVCONV_OPT_WARP_CHANNEL_SPLIT) != 0;
     auto kern = ring ? warp_wavefront_kernel<C, K, BWD, true, true, true>
                      : (pl.glb ? warp_wavefront_kernel<C, K, BWD, true, true>
                                : (pl.nb > 1 ? warp_wavefront_kernel<C, K, BWD, true> : warp_wavefront_kernel<C, K, BWD, false>));
@@ -157,7 +159,7 @@ int launch_warp_ck(const WarpPlan& pl, WarpParams prm, cudaStream_t st)
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = g_use_pdl.load() ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = opt(INVCONV_OPT_DEPENDENT_LAUNCH) ? 1 : 0;
     cfg.attrs = attr; cfg.numAttrs = 1;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
     if (e != cudaSuccess) {
@@ -183,13 +185,13 @@ GradWSmallPlan gradw_small_plan(int B, int C, int H, int W, int k)
 // the separate kernel against riding along: 18 us against 10 us (C=3, 32x32, k=3, batch 128), 11 us against
 // 4 us (C=1, 28x28, k=3, batch 256), 13 us against 118 us (C=3, 64x64, k=5, batch 16, where the sums do not
 // fit the wavefront's registers), 24 us against 75 us (C=1, 256x256, k=5, batch 4, images in global memory).
-// So it is used where the sums do not fit the registers or the images stay in global memory.  INVCONV_GW_SEPARATE=0/1 overrides (measurement knob).
+// So it is used where the sums do not fit the registers or the images stay in global memory (INVCONV_OPT_GRADW_SEPARATE overrides).
 bool gradw_separate(const WarpPlan& pl, const GradWSmallPlan& gs, int C, int k)
 {
     if (!gs.ok) return false;
-    const char* knob = std::getenv("INVCONV_GW_SEPARATE");      // read per call so that tests can switch it
-    if (knob && knob[0] == '0') return false;
-    if (knob && knob[0] == '1') return true;
+    const int knob = opt(INVCONV_OPT_GRADW_SEPARATE);
+    if (knob == 0) return false;
+    if (knob == 1) return true;
     return pl.glb || C * C * k * k > 81;
 }
 
@@ -206,7 +208,7 @@ int launch_gradw_small_ck(const GradWSmallPlan& gs, const GradWSmallParams& prm,
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = g_use_pdl.load() ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = opt(INVCONV_OPT_DEPENDENT_LAUNCH) ? 1 : 0;
     cfg.attrs = attr; cfg.numAttrs = 1;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
     if (e != cudaSuccess) {
@@ -367,7 +369,7 @@ namespace {
 TeamPlan team_plan(int B, int C, int H, int W, int k)
 {
     if (team_solve_smem(C, k) > kMaxDynSmem) return TeamPlan{};
-    return plan_team(B > 0 ? B : 1, C, H, W, k, kMaxDynSmem, sm_count());
+    return plan_team(B > 0 ? B : 1, C, H, W, k, kMaxDynSmem, sm_count(), opt(INVCONV_OPT_TEAM_VARIANT), opt(INVCONV_OPT_TEAM_CLUSTER));
 }
 
 GradWPlan gradw_plan(int B, int C, int H, int W, int k)
@@ -430,10 +432,9 @@ int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, c
     prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W; prm.nbc = gp.nbc; prm.tiles = gp.tiles; prm.plane = gp.plane;
     int rc = INVCONV_UNSUPPORTED;
     // tensor pipe (TF32 inputs) where the fragments line up: rows of whole 8-pixel chunks, conflict-free planes
-    const char* knob = std::getenv("INVCONV_GW_MMA");
     // (measured, kernel + reduction: 31 / 58 us against 41 / 87 us for the FMA kernel on the 48-channel shapes,
     // k = 3 / 5; 19 us against 25 us on the 12-channel one with all taps in one CTA)
-    const bool mma = g.W % 8 == 0 && gp.plane % 32 == 4 && !(knob && knob[0] == '0');
+    const bool mma = g.W % 8 == 0 && gp.plane % 32 == 4 && opt(INVCONV_OPT_GRADW_TENSOR_PIPE) != 0;
     int shares = gp.nbc;
     if (mma && gp.TC == 1) {                 // tiles of 16 channels: one CTA covers all taps, its own share count
         shares = gp.nbc_all;
@@ -473,7 +474,7 @@ int launch_team_inst(const TeamPlan& pl, const TeamParams& prm, cudaStream_t st)
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = pl.R; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = g_use_pdl.load() ? 1 : 0;
+    attr[1].val.programmaticStreamSerializationAllowed = opt(INVCONV_OPT_DEPENDENT_LAUNCH) ? 1 : 0;
     cfg.attrs = attr; cfg.numAttrs = 2;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
     if (e != cudaSuccess) {
@@ -499,7 +500,7 @@ int launch_pixel_inst(const TeamPlan& pl, const TeamParams& prm, cudaStream_t st
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = pl.R; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = g_use_pdl.load() ? 1 : 0;
+    attr[1].val.programmaticStreamSerializationAllowed = opt(INVCONV_OPT_DEPENDENT_LAUNCH) ? 1 : 0;
     cfg.attrs = attr; cfg.numAttrs = 2;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
     if (e != cudaSuccess) {
@@ -594,7 +595,7 @@ int launch_gradw_tensor(const float* gy, const float* x, float* gw, Geom g, void
 {
     const GradWTensorPlan gt = gradw_tensor_plan(g.B, g.C, g.H, g.W, g.k);
     const bool aligned = ((reinterpret_cast<uintptr_t>(gy) | reinterpret_cast<uintptr_t>(x)) & 15) == 0;
-    if (!gt.ok || !aligned || g.B == 0) return launch_gradw(gy, x, gw, g, ws, st);
+    if (!gt.ok || !aligned || g.B == 0 || opt(INVCONV_OPT_GRADW_TENSOR_PIPE) == 0) return launch_gradw(gy, x, gw, g, ws, st);
     float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + tensor_gradw_offset(g.B, g.C, g.H, g.W, g.k));
     const int rc = invconv_internal::gradw_tensor_launch(gt, gy, x, partials, g, st);
     if (rc) return rc;
@@ -904,8 +905,16 @@ int invconv_step_host(const float* y_host, const float* w_host, const float* gra
         cudaMemcpyAsync(d_gx, grad_x_host, act_b, cudaMemcpyHostToDevice, side->side);
         cudaEventRecord(side->gx_in, side->side);
     }
+    // on an error the side stream is still joined back into `stream`, so the caller's stream orders everything
+    auto fail = [&](int code) {
+        if (act_b) {
+            cudaEventRecord(side->x_out, side->side);
+            cudaStreamWaitEvent(st, side->x_out, 0);
+        }
+        return code;
+    };
     int r = invconv_forward_ws(d_y, d_w, d_x, B, C, H, W, k, ws, ws_b, stream);
-    if (r) return r;
+    if (r) return fail(r);
     if (act_b) {
         cudaEventRecord(side->x_ready, st);
         cudaStreamWaitEvent(side->side, side->x_ready, 0);
@@ -914,9 +923,9 @@ int invconv_step_host(const float* y_host, const float* w_host, const float* gra
         cudaStreamWaitEvent(st, side->gx_in, 0);
     }
     r = invconv_backward_ws(d_gx, d_x, d_w, d_gy, d_gw, B, C, H, W, k, ws, ws_b, stream);
-    if (r) return r;
+    if (r) return fail(r);
     r = invconv_logdet(d_w, d_ld, C, H, W, k, stream);
-    if (r) return r;
+    if (r) return fail(r);
     if (act_b) cudaMemcpyAsync(grad_y_host, d_gy, act_b, cudaMemcpyDeviceToHost, st);
     cudaMemcpyAsync(grad_w_host, d_gw, w_b, cudaMemcpyDeviceToHost, st);
     cudaMemcpyAsync(logdet_host, d_ld, sizeof(float), cudaMemcpyDeviceToHost, st);
@@ -978,6 +987,19 @@ int invconv_set_path(int path)
     return g_forced_path.exchange(path);
 }
 
+int invconv_set_option(int option, int value)
+{
+    if (option < 0 || option >= INVCONV_OPT_COUNT) return -1;
+    return g_opt[option].exchange(value);
+}
+
+int invconv_selftest_wait_timeout(unsigned limit_cycles, void* stream)
+{
+    if (limit_cycles < 1 || limit_cycles > (1u << 24)) return INVCONV_BAD_ARG;
+    probe_wait_timeout<<<1, 64, 0, as_stream(stream)>>>(limit_cycles);
+    return check_launch();
+}
+
 int invconv_path_for(int B, int C, int H, int W, int k)
 {
     if (check_shape(B, C, H, W, k) != INVCONV_OK) return -1;
@@ -1016,9 +1038,6 @@ int invconv_probe_step_latency(int mechanism, int steps, unsigned long long* cyc
     switch (mechanism) {
     case 0: probe_shuffle_chain<<<1, 32, 0, st>>>(steps, cycles_out); break;
     case 1: probe_smem_chain<<<1, 256, 0, st>>>(steps, cycles_out); break;
-    case 3: probe_fma_chain<<<1, 32, 0, st>>>(steps, cycles_out); break;
-    case 4: probe_group_chain<<<1, 256, 0, st>>>(steps, cycles_out); break;
-    case 5: probe_step_c3k3<<<1, 32, 0, st>>>(steps, cycles_out); break;
     case 2: {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2); cfg.blockDim = dim3(128); cfg.stream = st;

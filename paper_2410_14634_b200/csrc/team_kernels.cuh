@@ -194,12 +194,6 @@ struct TeamParams {
     int ncl;            // clusters in the grid
 };
 
-// Phase timing for development builds (-DINVCONV_TEAM_TIMING): thread 0 of CTA 0 prints SM-clock totals per phase.
-#ifdef INVCONV_TEAM_TIMING
-#define TEAM_TT(i) do { if (tid == 0) { const long long now_ = clock64(); tacc_[i] += now_ - tlast_; tlast_ = now_; } } while (0)
-#else
-#define TEAM_TT(i) do { } while (0)
-#endif
 
 __device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
@@ -240,9 +234,7 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
 {
     extern __shared__ __align__(128) float smem[];
     __shared__ unsigned long long bars[2];
-#ifdef INVCONV_TEAM_TIMING
-    const long long tstart_ = clock64();
-#endif
+    __shared__ int gave_up_flag;                   // a bounded wait of this CTA ran out: later waits no longer block
     const int C = p.C, H = p.H, W = p.W, K = p.K, CS = p.CS, R = p.R, CA = p.CA;
     const int HP = H + K - 1, WP = W + K - 1, HW = H * W;
     const int IMG = HP * WP * CS;
@@ -264,7 +256,7 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
 
     // Set-up that needs no global memory runs first, so that under programmatic dependent launch it overlaps
     // the kernel-transform kernel that precedes this one on the stream; griddepcontrol.wait then waits for it.
-    if (tid == 0) { mbar_init(&bars[0], NT >> 5); mbar_init(&bars[1], NT >> 5); fence_mbar_init(); }   // one arrival per warp
+    if (tid == 0) { gave_up_flag = 0; mbar_init(&bars[0], NT >> 5); mbar_init(&bars[1], NT >> 5); fence_mbar_init(); }   // one arrival per warp
     for (int i = tid; i < 2 * IMG; i += NT) smem[i] = 0.f;     // zero padding (and the channel padding) once
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -317,17 +309,11 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
     const int finq_i0 = tid / CAQ, finq_a0 = tid - finq_i0 * CAQ;
     const int finq_di = NT / CAQ, finq_da = NT - finq_di * CAQ;
 
-#ifdef INVCONV_TEAM_TIMING
-    long long tacc_[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    long long tlast_ = clock64();
-    if (threadIdx.x == 0 && blockIdx.x == 0) printf("team setup: %lld cycles\n", tlast_ - tstart_);
-#endif
     const int ND = H + W - 1;
     const int nq4 = HW >> 2;
     unsigned stepno = 0;                            // diagonals processed so far by this CTA, across images
-    bool alive = true;
-    for (int n = cl; n < p.B && alive; n += p.ncl) {
-        TEAM_TT(7);
+    volatile int* gave_up = &gave_up_flag;
+    for (int n = cl; n < p.B; n += p.ncl) {
         // right-hand side of this image, all channels, rotated for the transposed solve; the loads go out in
         // batches of eight requests per thread so that their latency is paid once per batch
         const float* src = p.rhs + (size_t)n * C * HW;
@@ -373,7 +359,6 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
             }
         }
         __syncthreads();
-        TEAM_TT(0);
 
         for (int d = 0; d < ND; ++d, ++stepno) {
             const int hlo = max(0, d - (W - 1));
@@ -414,13 +399,11 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
                             }
                 }
             }
-            TEAM_TT(1);
             // the previous diagonal: published by this CTA's threads and by the peers
             if (d > 0) {
                 const unsigned prev = stepno - 1u;
-                if (!mbar_wait_bounded(&bars[prev & 1u], (prev >> 1) & 1u)) alive = false;
+                mbar_wait_or_give_up(&bars[prev & 1u], (prev >> 1) & 1u, gave_up);
             }
-            TEAM_TT(2);
             // the two taps that read diagonal d-1
 #pragma unroll
             for (int q = 0; q < PM; q += 2) {
@@ -493,9 +476,7 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
                 else if (LG == 8) fold_rounds(std::integral_constant<int, 4>{});
                 else fold_rounds(std::integral_constant<int, 8>{});
             }
-            TEAM_TT(3);
             __syncthreads();
-            TEAM_TT(4);
             // finish the diagonal: sum the warps' partial sums and publish to every CTA of the cluster
             unsigned long long* mybar = &bars[stepno & 1u];
             if (R > 1 && tid == 0) mbar_expect_tx_only(mybar, (unsigned)((R - 1) * npix * CA * 4));
@@ -550,13 +531,11 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
             }
             __syncwarp();
             if ((tid & 31) == 0) mbar_arrive(mybar);      // the warp's stores are ordered before its one arrival
-            TEAM_TT(5);
         }
         {   // the last diagonal
             const unsigned prev = stepno - 1u;
-            if (!mbar_wait_bounded(&bars[prev & 1u], (prev >> 1) & 1u)) alive = false;
+            mbar_wait_or_give_up(&bars[prev & 1u], (prev >> 1) & 1u, gave_up);
         }
-        TEAM_TT(6);
         // write back this CTA's channels
         float* dst = p.out + (size_t)n * C * HW + (size_t)r * CA * HW;
         if (p.vec) {
@@ -583,14 +562,8 @@ __global__ void __launch_bounds__(MAXT) team_wavefront_kernel(TeamParams p)
         // nobody publishes the next image's first diagonal into an image that is still being written back
         if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
     }
-    if (!alive && tid == 0) raise_status(INVCONV_TIMEOUT);
+    if (tid == 0 && *gave_up) raise_status(INVCONV_TIMEOUT);
     if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); }   // no CTA exits while peers may still store into it
-#ifdef INVCONV_TEAM_TIMING
-    TEAM_TT(7);
-    if (tid == 0 && blockIdx.x == 0)
-        printf("team timing (cycles): load %lld | noncrit %lld | wait %lld | crit+red %lld | bar %lld | finalize %lld | lastwait %lld | store %lld\n",
-               tacc_[0], tacc_[1], tacc_[2], tacc_[3], tacc_[4], tacc_[5], tacc_[6], tacc_[7]);
-#endif
 }
 
 // ---------------------------------------------------------------------------
@@ -616,6 +589,7 @@ __global__ void __launch_bounds__(256, (NGN <= 3 ? 2 : 1)) team_pixel_kernel(Tea
 {
     extern __shared__ __align__(128) float smem[];
     __shared__ unsigned long long bars[2];
+    __shared__ int gave_up_flag;                   // a bounded wait of this CTA ran out: later waits no longer block
     const int C = p.C, H = p.H, W = p.W, K = p.K, CS = p.CS, R = p.R, CA = p.CA;
     const int HP = H + K - 1, WP = W + K - 1, HW = H * W;
     const int IMG = HP * WP * CS;
@@ -635,7 +609,7 @@ __global__ void __launch_bounds__(256, (NGN <= 3 ? 2 : 1)) team_pixel_kernel(Tea
     const int GN = (K > 1 ? K * K - 2 : 1) * CB4, GC = (K > 1 ? 2 : 0) * CB4;
     const int DS = (WP - 1) * CS;
 
-    if (tid == 0) { mbar_init(&bars[0], NTEAM); mbar_init(&bars[1], NTEAM); fence_mbar_init(); }   // one arrival per team
+    if (tid == 0) { gave_up_flag = 0; mbar_init(&bars[0], NTEAM); mbar_init(&bars[1], NTEAM); fence_mbar_init(); }   // one arrival per team
     for (int i = tid; i < 2 * IMG; i += NT) smem[i] = 0.f;
     asm volatile("griddepcontrol.wait;" ::: "memory");          // the kernel transform before us has completed
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -682,8 +656,8 @@ __global__ void __launch_bounds__(256, (NGN <= 3 ? 2 : 1)) team_pixel_kernel(Tea
     const int ND = H + W - 1;
     const int nq4 = HW >> 2;
     unsigned stepno = 0;
-    bool alive = true;
-    for (int n = cl; n < p.B && alive; n += p.ncl) {
+    volatile int* gave_up = &gave_up_flag;
+    for (int n = cl; n < p.B; n += p.ncl) {
         const float* src = p.rhs + (size_t)n * C * HW;
         if (p.vec) {
             const float4* src4 = reinterpret_cast<const float4*>(src);
@@ -765,7 +739,7 @@ __global__ void __launch_bounds__(256, (NGN <= 3 ? 2 : 1)) team_pixel_kernel(Tea
                 __syncthreads();
             } else if (d > 0) {
                 const unsigned prev = stepno - 1u;
-                if (!mbar_wait_bounded(&bars[prev & 1u], (prev >> 1) & 1u)) alive = false;
+                mbar_wait_or_give_up(&bars[prev & 1u], (prev >> 1) & 1u, gave_up);
             }
             unsigned long long* mybar = &bars[stepno & 1u];
             if (R > 1 && tid == 0) mbar_expect_tx_only(mybar, (unsigned)((R - 1) * npix * CA * 4));
@@ -841,7 +815,7 @@ __global__ void __launch_bounds__(256, (NGN <= 3 ? 2 : 1)) team_pixel_kernel(Tea
         }
         if (R > 1) {
             const unsigned prev = stepno - 1u;
-            if (!mbar_wait_bounded(&bars[prev & 1u], (prev >> 1) & 1u)) alive = false;
+            mbar_wait_or_give_up(&bars[prev & 1u], (prev >> 1) & 1u, gave_up);
         }
         __syncthreads();
         float* dst = p.out + (size_t)n * C * HW + (size_t)r * CA * HW;
@@ -868,7 +842,7 @@ __global__ void __launch_bounds__(256, (NGN <= 3 ? 2 : 1)) team_pixel_kernel(Tea
         }
         if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
     }
-    if (!alive && tid == 0) raise_status(INVCONV_TIMEOUT);
+    if (tid == 0 && *gave_up) raise_status(INVCONV_TIMEOUT);
     if (R > 1) { cluster_arrive_release(); cluster_wait_acquire(); }
 }
 
@@ -885,7 +859,7 @@ struct TeamPlan {
 };
 
 // Pixel-team variant: smallest estimated time over cluster size and warps per team.
-inline TeamPlan plan_team_pixel(int B, int C, int H, int W, int K, size_t max_smem, int sm_count)
+inline TeamPlan plan_team_pixel(int B, int C, int H, int W, int K, size_t max_smem, int sm_count, bool forced = false)
 {
     TeamPlan best;
     double best_cost = 1e30;
@@ -899,9 +873,8 @@ inline TeamPlan plan_team_pixel(int B, int C, int H, int W, int K, size_t max_sm
     const int menu[3][2] = {{3, 1}, {6, 2}, {12, 3}};
     // Measured on B200: across a cluster the slice variant is faster (wide48_k3: 108 us vs 181 us), for images
     // that one CTA serves the pixel teams are (cifar_sq: 41 us vs 72 us); so only R = 1 is planned here unless
-    // the measurement knob asks for more.
-    const char* variant = getenv("INVCONV_TEAM_VARIANT");
-    const int rmax = (variant && variant[0] == 'p') ? 8 : 1;
+    // the variant is forced (a measurement control).
+    const int rmax = forced ? 8 : 1;
     for (int R = 1; R <= rmax; R *= 2) {
         if (C % R != 0) continue;
         const int CA = C / R;
@@ -948,13 +921,14 @@ inline TeamPlan plan_team_pixel(int B, int C, int H, int W, int K, size_t max_sm
     return best;
 }
 
-inline TeamPlan plan_team(int B, int C, int H, int W, int K, size_t max_smem, int sm_count)
+// variant: 0 by shape, 1 channel-slice kernel, 2 pixel-team kernel; forced_r: 0 by shape, else the cluster size
+// of the channel-slice kernel (test and measurement controls).
+inline TeamPlan plan_team(int B, int C, int H, int W, int K, size_t max_smem, int sm_count, int variant = 0, int forced_r = 0)
 {
     TeamPlan best;
     if (C < 1 || K < 1) return best;
-    const char* variant = getenv("INVCONV_TEAM_VARIANT");       // measurement knob: "slice" or "pixel"
-    if (!variant || variant[0] != 's') {
-        const TeamPlan px = plan_team_pixel(B, C, H, W, K, max_smem, sm_count);
+    if (variant != 1) {
+        const TeamPlan px = plan_team_pixel(B, C, H, W, K, max_smem, sm_count, variant == 2);
         if (px.ok) return px;
     }
     // cluster size: enough CTAs that the kernel's share fits one CTA's registers, then fill the SMs
@@ -963,10 +937,7 @@ inline TeamPlan plan_team(int B, int C, int H, int W, int K, size_t max_smem, in
     while (R < 8 && (long long)C * C * K * K / R > 30000 && divisible(R * 2)) R *= 2;
     if ((long long)C * C * K * K / R > 30000) return best;
     while (R < 8 && (long long)B * R * 2 <= sm_count && divisible(R * 2)) R *= 2;
-    if (const char* e = getenv("INVCONV_TEAM_R")) {           // measurement knob: force the cluster size
-        const int rr = atoi(e);
-        if (rr >= 1 && rr <= 8 && C % rr == 0) R = rr;
-    }
+    if (forced_r >= 1 && forced_r <= 8 && C % forced_r == 0) R = forced_r;
     const int CA = C / R;
     const int CB4 = (C + 3) / 4;
     int CS = CB4 * 4;

@@ -72,7 +72,7 @@ namespace tensor_detail {
 #define TENSOR_TT(i) do { } while (0)
 #endif
 
-constexpr long long kWaitLimit = 1ll << 27;      // SM cycles (about 70 ms) before a wait gives up
+constexpr long long kWaitLimit = 1ll << 24;      // SM cycles (about 8 ms) before a wait gives up
 
 // Waits for the phase of `bar` with the given parity; returns at once when the CTA has already given up.
 __device__ __forceinline__ void wait_bar(unsigned long long* bar, unsigned parity, volatile int* gave_up)

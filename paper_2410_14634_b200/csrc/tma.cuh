@@ -49,6 +49,20 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsig
     return true;
 }
 
+// Bounded wait for kernels whose control flow must stay uniform when a wait gives up: `gave_up` is a flag in
+// the CTA's shared memory.  The first wait that runs out (about 8 ms of SM clock) sets it; from then on no
+// wait of the CTA blocks.  Callers keep running through all of their barriers and report the flag at the end.
+__device__ __forceinline__ void mbar_wait_or_give_up(unsigned long long* bar, unsigned parity, volatile int* gave_up)
+{
+    if (mbar_try_wait(bar, parity)) return;
+    if (*gave_up) return;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*gave_up) return;
+        if (clock64() - t0 > (1ll << 24)) { *gave_up = 1; return; }
+    }
+}
+
 // global -> shared, completion counted in bytes on `bar`.
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, unsigned bytes, unsigned long long* bar)
 {

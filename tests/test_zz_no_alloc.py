@@ -5,7 +5,9 @@ inside another framework -- must not call an allocator once they are running.
 `invconv_backward_noalloc` serves them: every buffer comes from the caller and
 the library's own scratch is a fixed array inside the library image.  This test
 calls it through the C ABI and checks it against the workspace-taking entry
-point, twice in a row (the shared scratch must be left reusable).
+point and against the float64 oracle, twice in a row (the shared scratch must
+be left reusable), and checks that the device's free memory does not move
+across the second call (the first call of a shape may load kernel code).
 
 The file name sorts last on purpose: a run that stops at the first failure has
 then already run every other test.
@@ -33,18 +35,28 @@ def test_noalloc_backward_matches_workspace_backward_twice():
         x = binding.invconv_forward(yd, wd)
         gy_ref, gw_ref = binding.invconv_backward(gxd, x, wd)          # existing entry point (caller's workspace)
         torch.cuda.synchronize()
+        from oracle import api as oracle
+        gy_o, gw_o = oracle.invconv_backward(gx, x.cpu().numpy().astype(np.float64), w)
         st = torch.cuda.current_stream().cuda_stream
+        free_before = None
         for attempt in range(2):                                       # two calls in a row share the fixed scratch
             gy = torch.full_like(gxd, float("nan"))
             gw = torch.full_like(wd, float("nan"))
+            if attempt == 1:
+                torch.cuda.synchronize()
+                free_before = torch.cuda.mem_get_info()[0]
             rc = L.invconv_backward_noalloc(gxd.data_ptr(), x.data_ptr(), wd.data_ptr(), gy.data_ptr(), gw.data_ptr(),
                                             B, s.C, s.H, s.W, s.k, ctypes.c_void_p(st))
             assert rc == binding.OK, (name, attempt, rc)
             torch.cuda.synchronize()
+            if attempt == 1:
+                assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
             assert binding.invconv_get_status() == 0
             assert nmax_err(gy.cpu().numpy(), gy_ref.cpu().numpy()) <= 1e-4, (name, attempt)
             assert nmax_err(gw.cpu().numpy(), gw_ref.cpu().numpy()) <= 1e-3, (name, attempt)
             assert torch.equal(gy, gy_ref) and torch.equal(gw, gw_ref)  # same kernel, same order of sums
+            assert nmax_err(gy.cpu().numpy(), gy_o) <= 1e-4, (name, attempt)
+            assert nmax_err(gw.cpu().numpy(), gw_o) <= 1e-3, (name, attempt)
 
 
 def test_noalloc_backward_rejects_what_it_cannot_serve():
