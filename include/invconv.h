@@ -121,6 +121,30 @@ int invconv_backward_logdet(const float* grad_x, const float* x, const float* w,
                             float* grad_y, float* grad_w,
                             int B, int C, int H, int W, int k, void* stream);
 
+/* The layer inside one step of the paper's Inverse-Flow model (Section 4, Fig. 3: Inv-Conv, then Actnorm,
+ * then a 1x1 convolution), with the two neighbours folded into the layer's calls.  Both neighbours act on one
+ * pixel at a time:
+ *     z[n,c,h,w] = s[c] * x[n,c,h,w] + b[c]            Actnorm (per-channel affine map)
+ *     u[n,o,h,w] = sum_c V[o][c] * z[n,c,h,w]          1x1 convolution (C x C channel mix)
+ *
+ * invconv_flow_step_forward:  x = f^{-1}(y) (saved for the backward pass) and u = V (s * x + b).
+ *   y in; w [C,C,k,k], s [C], b [C], V [C][C] in; x, u [B,C,H,W] out; logdet: ONE device float or NULL,
+ *   the step's log-determinant  H*W * ( -sum_c log|w[c][c][k-1][k-1]| + sum_c log|s[c]| + log|det V| )
+ *   (accumulated in double; det V by Gaussian elimination with partial pivoting).
+ * invconv_flow_step_backward: given grad_u (gradient of the loss with respect to u) and the saved x,
+ *   grad_y = M^{-T} ( s * V^T grad_u ),  grad_w as in invconv_backward,
+ *   grad_V[o][c] = sum grad_u[n,o,h,w] * z[n,c,h,w],  grad_s[c] = sum (V^T grad_u)[n,c,h,w] * x[n,c,h,w],
+ *   grad_b[c] = sum (V^T grad_u)[n,c,h,w]   (sums over batch and pixels, fixed order).  All outputs non-NULL.
+ * For shapes of the warp-shuffle family whose images fit shared memory the neighbours are applied inside the
+ * wavefront kernel (u is written while x is stored; the incoming gradient is transformed as it is loaded);
+ * other shapes run the layer's kernels and per-pixel kernels one after the other -- same results.  Scratch
+ * comes from the device's stream-ordered memory pool.  Argument rules and errors as for invconv_forward. */
+int invconv_flow_step_forward(const float* y, const float* w, const float* s, const float* b, const float* V,
+                              float* x, float* u, float* logdet, int B, int C, int H, int W, int k, void* stream);
+int invconv_flow_step_backward(const float* grad_u, const float* x, const float* w, const float* s, const float* b,
+                               const float* V, float* grad_y, float* grad_w, float* grad_s, float* grad_b, float* grad_V,
+                               int B, int C, int H, int W, int k, void* stream);
+
 /* Scratch bytes a forward or backward call of this shape needs (0 if none).
  * Same value for both directions. */
 size_t invconv_workspace_bytes(int B, int C, int H, int W, int k);

@@ -46,6 +46,10 @@ def lib() -> ctypes.CDLL:
         L.invconv_logdet.argtypes = [fp, fp, ci, ci, ci, ci, vp]
         L.invconv_forward_logdet.argtypes = [fp, fp, fp, fp, ci, ci, ci, ci, ci, vp]
         L.invconv_backward_logdet.argtypes = [fp, fp, fp, fp, fp, fp, ci, ci, ci, ci, ci, vp]
+        L.invconv_flow_step_forward.argtypes = [fp] * 8 + [ci] * 5 + [vp]
+        L.invconv_flow_step_forward.restype = ci
+        L.invconv_flow_step_backward.argtypes = [fp] * 11 + [ci] * 5 + [vp]
+        L.invconv_flow_step_backward.restype = ci
         L.invconv_workspace_bytes.argtypes = [ci] * 5
         L.invconv_workspace_bytes.restype = sz
         L.invconv_forward_ws.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, vp, sz, vp]
@@ -234,6 +238,38 @@ def invconv_backward_logdet(grad_x: torch.Tensor, x: torch.Tensor, w: torch.Tens
                                              gy.data_ptr(), gw.data_ptr(), B, C, H, W, k,
                                              _stream_ptr(stream, x.device)), "invconv_backward_logdet")
     return gy, gw
+
+
+def invconv_flow_step_forward(y: torch.Tensor, w: torch.Tensor, s: torch.Tensor, b: torch.Tensor, V: torch.Tensor,
+                              want_logdet: bool = True, stream: Optional[torch.cuda.Stream] = None):
+    """(x, u, logdet) of one flow step: x = f^{-1}(y), u = V (s * x + b); logdet is a one-element tensor or None."""
+    _act(y, "y")
+    B, C, H, W = y.shape
+    k = _kern(w, C)
+    x, u = torch.empty_like(y), torch.empty_like(y)
+    ld = torch.empty(1, dtype=torch.float32, device=y.device) if want_logdet else None
+    with torch.cuda.device(y.device):
+        _check(lib().invconv_flow_step_forward(y.data_ptr(), w.data_ptr(), s.data_ptr(), b.data_ptr(), V.data_ptr(),
+                                               x.data_ptr(), u.data_ptr(), ld.data_ptr() if ld is not None else None,
+                                               B, C, H, W, k, _stream_ptr(stream, y.device)), "invconv_flow_step_forward")
+    return x, u, ld
+
+
+def invconv_flow_step_backward(grad_u: torch.Tensor, x: torch.Tensor, w: torch.Tensor, s: torch.Tensor, b: torch.Tensor,
+                               V: torch.Tensor, stream: Optional[torch.cuda.Stream] = None):
+    """(grad_y, grad_w, grad_s, grad_b, grad_V) through one flow step, given grad_u and the saved x."""
+    _act(grad_u, "grad_u")
+    _act(x, "x")
+    B, C, H, W = x.shape
+    k = _kern(w, C)
+    gy, gw = torch.empty_like(x), torch.empty_like(w)
+    gs, gb, gV = torch.empty_like(s), torch.empty_like(b), torch.empty_like(V)
+    with torch.cuda.device(x.device):
+        _check(lib().invconv_flow_step_backward(grad_u.data_ptr(), x.data_ptr(), w.data_ptr(), s.data_ptr(), b.data_ptr(),
+                                                V.data_ptr(), gy.data_ptr(), gw.data_ptr(), gs.data_ptr(), gb.data_ptr(),
+                                                gV.data_ptr(), B, C, H, W, k, _stream_ptr(stream, x.device)),
+               "invconv_flow_step_backward")
+    return gy, gw, gs, gb, gV
 
 
 class HostStep:

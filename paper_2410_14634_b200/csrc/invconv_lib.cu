@@ -241,11 +241,19 @@ int launch_gradw_small(const GradWSmallPlan& gs, const float* gy, const float* x
     return INVCONV_UNSUPPORTED;
 }
 
+// The per-pixel neighbours of the layer in a flow step, applied inside the wavefront kernel (see WarpParams).
+struct WarpMix {
+    const float* V = nullptr; const float* s = nullptr; const float* b = nullptr;
+    float* u_out = nullptr;     // forward
+    bool grad_in = false;       // backward
+};
+
 int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const float* xsaved, float* gw, Geom g,
-                void* ws, cudaStream_t st)
+                void* ws, cudaStream_t st, const WarpMix* mix = nullptr)
 {
     const WarpPlan pl = plan_warp(g.B, g.C, g.H, g.W, g.k, bwd);
     if (!pl.ok) return INVCONV_UNSUPPORTED;
+    if (mix && pl.glb) return INVCONV_UNSUPPORTED;       // images in global memory: the caller composes the step
     const GradWSmallPlan gs = (bwd && gw) ? gradw_small_plan(g.B, g.C, g.H, g.W, g.k) : GradWSmallPlan{};
     const bool separate = bwd && gw && ws && gradw_separate(pl, gs, g.C, g.k);
     WarpParams prm;
@@ -253,6 +261,11 @@ int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const fl
     prm.counter = static_cast<unsigned*>(ws);
     prm.partials = ws ? reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES) : nullptr;
     prm.B = g.B; prm.H = g.H; prm.W = g.W; prm.nb = pl.nb; prm.ipc = pl.ipc;
+    if (mix) {
+        prm.mix_V = mix->V; prm.mix_s = mix->s; prm.mix_b = mix->b;
+        prm.mix_out = bwd ? nullptr : mix->u_out;
+        prm.mix_in = (bwd && mix->grad_in) ? 1 : 0;
+    }
     const size_t chw = (size_t)g.C * g.H * g.W;
     const bool aligned = ((reinterpret_cast<uintptr_t>(rhs) | reinterpret_cast<uintptr_t>(out) |
                            reinterpret_cast<uintptr_t>(xsaved)) & 15) == 0;
@@ -743,6 +756,30 @@ StepSide* step_side()
 }
 
 }  // namespace
+
+namespace invconv_internal {
+
+// The layer with its flow-step neighbours inside the warp-family kernel; INVCONV_UNSUPPORTED where that family
+// (or its shared-memory mode) does not serve the shape -- the caller then composes the step from separate kernels.
+int warp_step_forward(const float* y, const float* w, const float* s, const float* b, const float* V, float* x, float* u,
+                      Geom g, void* ws, cudaStream_t st)
+{
+    if (resolve_path(g.B, g.C, g.H, g.W, g.k) != INVCONV_PATH_WARP) return INVCONV_UNSUPPORTED;
+    WarpMix mix;
+    mix.V = V; mix.s = s; mix.b = b; mix.u_out = u;
+    return launch_warp(false, y, w, x, nullptr, nullptr, g, ws, st, &mix);
+}
+
+int warp_step_backward(const float* grad_u, const float* x, const float* w, const float* s, const float* V,
+                       float* grad_y, float* grad_w, Geom g, void* ws, cudaStream_t st)
+{
+    if (resolve_path(g.B, g.C, g.H, g.W, g.k) != INVCONV_PATH_WARP) return INVCONV_UNSUPPORTED;
+    WarpMix mix;
+    mix.V = V; mix.s = s; mix.grad_in = true;
+    return launch_warp(true, grad_u, w, grad_y, x, grad_w, g, ws, st, &mix);
+}
+
+}  // namespace invconv_internal
 
 extern "C" {
 

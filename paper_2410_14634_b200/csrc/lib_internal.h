@@ -29,6 +29,13 @@ inline int set_smem_limit(Kern kern, size_t smem)
     return INVCONV_OK;
 }
 
+// invconv_lib.cu: forward / backward of the layer with Actnorm and the 1x1 convolution applied inside the warp-family
+// kernel (see flow_step_lib.cu); INVCONV_UNSUPPORTED where that kernel does not serve the shape.
+int warp_step_forward(const float* y, const float* w, const float* s, const float* b, const float* V, float* x, float* u,
+                      invconv::Geom g, void* ws, cudaStream_t st);
+int warp_step_backward(const float* grad_u, const float* x, const float* w, const float* s, const float* V,
+                       float* grad_y, float* grad_w, invconv::Geom g, void* ws, cudaStream_t st);
+
 // tensor_lib.cu: the tcgen05 wavefront (kernel transform into A, operand packing into wop, solve).
 int tensor_launch(const invconv::TensorPlan& pl, bool bwd, const float* rhs, const float* w, float* out,
                   invconv::Geom g, float* A, unsigned char* wop, cudaStream_t st);

@@ -63,6 +63,13 @@ struct WarpParams {
     int bulk;              // images are 16-byte aligned multiples of 16 bytes
     int glb;               // images stay in global memory (too large for shared memory)
     int vec;               // image rows are 16-byte aligned multiples of 16 bytes (ring mode: 16-byte copies)
+    // The per-pixel neighbours of the layer in a flow step (Actnorm z = s*x + b, then the 1x1 convolution
+    // u = V z), applied while the image is on chip; all nullptr = the plain layer.
+    const float* mix_V = nullptr;   // [C][C]
+    const float* mix_s = nullptr;   // [C]
+    const float* mix_b = nullptr;   // [C] (forward only)
+    float* mix_out = nullptr;       // forward: u [B][C][H][W], written beside x
+    int mix_in = 0;                 // backward: rhs holds grad_u; grad_x = s * (V^T grad_u) is formed after the load
 };
 
 template <int C> struct ColVec;
@@ -889,6 +896,35 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     if (has_img) {
         if (!GLB && p.bulk) ok = mbar_wait_bounded(&bars[li], 0);
         ok = __all_sync(0xffffffffu, ok);
+    }
+    if constexpr (BWD && !GLB) {
+        if (p.mix_in) {
+            // load prologue of the transposed solve: the incoming gradient of the 1x1 convolution's output becomes
+            // the gradient of x, pixel by pixel and in place: grad_x[c] = s[c] * sum_o V[o][c] * grad_u[o]
+            if (has_img && ok) {
+                float A[C][C];
+#pragma unroll
+                for (int c = 0; c < C; ++c)
+#pragma unroll
+                    for (int o = 0; o < C; ++o) A[c][o] = __ldg(p.mix_s + c) * __ldg(p.mix_V + o * C + c);
+                for (int i = j * 32 + lane; i < HW; i += p.nb * 32) {
+                    float g[C], r[C];
+#pragma unroll
+                    for (int o = 0; o < C; ++o) g[o] = img[o * HW + i];
+#pragma unroll
+                    for (int c = 0; c < C; ++c) {
+                        r[c] = 0.f;
+#pragma unroll
+                        for (int o = 0; o < C; ++o) r[c] = fmaf(A[c][o], g[o], r[c]);
+                    }
+#pragma unroll
+                    for (int c = 0; c < C; ++c) img[c * HW + i] = r[c];
+                }
+            }
+            __syncthreads();
+        }
+    }
+    if (has_img) {
         WARP_TT(2);
         if (ok) {
             if constexpr (CS)
@@ -925,6 +961,37 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
             }
         } else {
             for (int i = j * 32 + lane; i < CHW; i += p.nb * 32) dst[i] = img[i];
+        }
+    }
+
+    if constexpr (!BWD && !GLB) {
+        if (p.mix_out != nullptr && has_img) {
+            // store epilogue of the forward solve: Actnorm and the 1x1 convolution act on one pixel at a time, so
+            // u = V (s * x + b) is formed from the solved image while it is still in shared memory
+            float A[C][C], cb[C];
+#pragma unroll
+            for (int o = 0; o < C; ++o) {
+                cb[o] = 0.f;
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    const float v = __ldg(p.mix_V + o * C + c);
+                    A[o][c] = v * __ldg(p.mix_s + c);
+                    cb[o] = fmaf(v, __ldg(p.mix_b + c), cb[o]);
+                }
+            }
+            float* dst2 = p.mix_out + (size_t)n * CHW;
+            for (int i = j * 32 + lane; i < HW; i += p.nb * 32) {
+                float xin[C];
+#pragma unroll
+                for (int c = 0; c < C; ++c) xin[c] = img[c * HW + i];
+#pragma unroll
+                for (int o = 0; o < C; ++o) {
+                    float u = cb[o];
+#pragma unroll
+                    for (int c = 0; c < C; ++c) u = fmaf(A[o][c], xin[c], u);
+                    dst2[o * HW + i] = u;
+                }
+            }
         }
     }
 
