@@ -390,13 +390,22 @@ GradWPlan gradw_plan(int B, int C, int H, int W, int k)
     return plan_gradw(B, C, H, W, k, kMaxDynSmem / 2, sm_count());      // two CTAs per SM
 }
 
+GradWTensorPlan gradw_tensor_plan(int B, int C, int H, int W, int k)
+{
+    return plan_gradw_tensor(B > 0 ? B : 1, C, H, W, k, kMaxDynSmem, sm_count());
+}
+
+// Workspace of the team family: control words, transformed kernel, C*C floats, then the partial sums of
+// grad_w -- one set per batch share of whichever correlation kernel runs (the tcgen05 one included).
 size_t team_workspace_bytes(int B, int C, int H, int W, int k)
 {
     if (!team_plan(B, C, H, W, k).ok) return 0;
     const size_t na = sizeof(float) * (size_t)k * k * C * C;
     const GradWPlan gp = gradw_plan(B, C, H, W, k);
-    const int shares = gp.nbc > gp.nbc_all ? gp.nbc : gp.nbc_all;
-    return INVCONV_WS_CONTROL_BYTES + na + sizeof(float) * (size_t)C * C + (gp.ok ? na * shares : 0);
+    const GradWTensorPlan gt = gradw_tensor_plan(B, C, H, W, k);
+    int shares = gp.ok ? (gp.nbc > gp.nbc_all ? gp.nbc : gp.nbc_all) : 0;
+    if (gt.ok && gt.S > shares) shares = gt.S;
+    return INVCONV_WS_CONTROL_BYTES + na + sizeof(float) * (size_t)C * C + na * shares;
 }
 
 template <int TC, int K>
@@ -584,11 +593,6 @@ size_t tensor_wop_offset(int B, int C, int H, int W, int k)
     return (base + 255) & ~(size_t)255;
 }
 
-GradWTensorPlan gradw_tensor_plan(int B, int C, int H, int W, int k)
-{
-    return plan_gradw_tensor(B > 0 ? B : 1, C, H, W, k, kMaxDynSmem, sm_count());
-}
-
 size_t tensor_gradw_offset(int B, int C, int H, int W, int k)
 {
     return (tensor_wop_offset(B, C, H, W, k) + tensor_plan(B, C, H, W, k).wop_bytes + 255) & ~(size_t)255;
@@ -604,12 +608,13 @@ size_t tensor_workspace_bytes(int B, int C, int H, int W, int k)
 }
 
 // grad_w through the tensor-core correlation kernel and the fixed-order reduction over its shares.
-int launch_gradw_tensor(const float* gy, const float* x, float* gw, Geom g, void* ws, cudaStream_t st)
+// `partials_offset`: where in the workspace the [shares][k*k][C][C] partial sums go.
+int launch_gradw_tensor(const float* gy, const float* x, float* gw, Geom g, void* ws, size_t partials_offset, cudaStream_t st)
 {
     const GradWTensorPlan gt = gradw_tensor_plan(g.B, g.C, g.H, g.W, g.k);
     const bool aligned = ((reinterpret_cast<uintptr_t>(gy) | reinterpret_cast<uintptr_t>(x)) & 15) == 0;
     if (!gt.ok || !aligned || g.B == 0 || opt(INVCONV_OPT_GRADW_TENSOR_PIPE) == 0) return launch_gradw(gy, x, gw, g, ws, st);
-    float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + tensor_gradw_offset(g.B, g.C, g.H, g.W, g.k));
+    float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + partials_offset);
     const int rc = invconv_internal::gradw_tensor_launch(gt, gy, x, partials, g, st);
     if (rc) return rc;
     const size_t na = (size_t)g.k * g.k * g.C * g.C;
@@ -699,7 +704,10 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
             const int rc = launch_team(true, gx, w, gy, g, ws, st);
             if (rc) return rc;
         }
-        if (gw) return launch_gradw(gy, x, gw, g, ws, st);
+        if (gw) {
+            const size_t na = sizeof(float) * (size_t)g.k * g.k * g.C * g.C;
+            return launch_gradw_tensor(gy, x, gw, g, ws, INVCONV_WS_CONTROL_BYTES + na + sizeof(float) * (size_t)g.C * g.C, st);
+        }
         return INVCONV_OK;
     }
     case INVCONV_PATH_TENSOR: {
@@ -707,7 +715,7 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
             const int rc = launch_tensor(true, gx, w, gy, g, ws, st);
             if (rc) return rc;
         }
-        if (gw) return launch_gradw_tensor(gy, x, gw, g, ws, st);
+        if (gw) return launch_gradw_tensor(gy, x, gw, g, ws, tensor_gradw_offset(g.B, g.C, g.H, g.W, g.k), st);
         return INVCONV_OK;
     }
     default:
