@@ -267,6 +267,30 @@ def test_grad_w_many_channels_fma_and_tensor_pipe(B, oracle, shape, mma, family)
     assert rel <= (5e-3 if mma == 1 else 2e-4), rel
 
 
+@pytest.mark.parametrize("name", ["mnist", "cifar_sq", "wide48_k3"])
+def test_batch_shards_sum_to_the_full_grad_w(B, oracle, name):
+    """The multi-GPU partition on one GPU: images are independent and grad_w is a sum over the batch, so two
+    half-batches run one after the other give the full batch's x and grad_y and, summed, its grad_w (what the
+    all-reduce does across ranks)."""
+    import torch
+    from paper_2410_14634_b200 import sharding
+    s, w, y, gx = workloads.make(name)
+    wd = dev(w)
+    xs, gys, gw_sum = [], [], None
+    for rank in range(2):
+        start, count = sharding.shard_batch(s.B, 2, rank)
+        x = B.invconv_forward(dev(y[start:start + count]), wd)
+        gy, gw = B.invconv_backward(dev(gx[start:start + count]), x, wd)
+        xs.append(x); gys.append(gy)
+        gw_sum = gw.clone() if gw_sum is None else gw_sum + gw
+    torch.cuda.synchronize()
+    x_ref = oracle.invconv_forward(y, w)
+    gy_ref, gw_ref = oracle.invconv_backward(gx, x_ref, w)
+    assert nmax_err(torch.cat(xs).cpu().numpy(), x_ref) <= TOL_X
+    assert nmax_err(torch.cat(gys).cpu().numpy(), gy_ref) <= TOL_X
+    assert nmax_err(gw_sum.cpu().numpy(), gw_ref) <= TOL_GW
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_once_and_the_context_stays_usable(B, oracle):
     """The failure path of the device-side waits, without a fault: a probe kernel waits on a barrier that
     nothing completes, gives up after its limit, raises the status word and returns.  The status query reports
