@@ -113,8 +113,10 @@ int invconv_logdet(const float* w, float* logdet, int C, int H, int W, int k, vo
  *   other entry).  grad_logdet points to ONE device float (the upstream
  *   gradient of the loss with respect to the log-det value returned above);
  *   grad_w must be non-NULL here.
- * Argument rules, scratch and errors are those of invconv_forward/backward;
- * the extra work is one single-warp kernel launch per call. */
+ * Argument rules, scratch and errors are those of invconv_forward/backward.
+ * No extra launch: the log-det is written by a spare warp of the forward kernels (in the shadow of the image's
+ * arrival) and its term is added where the final grad_w is written; only the fallback kernels for shapes no
+ * specialised family serves use one single-warp launch more. */
 int invconv_forward_logdet(const float* y, const float* w, float* x, float* logdet,
                            int B, int C, int H, int W, int k, void* stream);
 int invconv_backward_logdet(const float* grad_x, const float* x, const float* w, const float* grad_logdet,

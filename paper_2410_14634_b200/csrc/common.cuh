@@ -35,6 +35,34 @@ __device__ __forceinline__ float tf32_hi(float v)
     return __uint_as_float(u);
 }
 
+// The log-det folded into the training step (Section 4: the layer's log-det enters the likelihood).
+// Forward: kernels that are given `out` write H*W*sum_c log|w[c][c][k-1][k-1]|, accumulated in double by one warp.
+// Backward: the kernels that write the final grad_w add  grad_logdet * H*W / w[c][c][k-1][k-1]  on the channel
+// diagonal of the tap that multiplies the pixel itself (tap index 0 in (dh, dw) order).
+struct LogdetFuse {
+    const float* grad_logdet = nullptr;   // one float: upstream gradient with respect to the log-det (nullptr: none)
+    const float* w = nullptr;             // [C][C][k][k]
+    int HW = 0;
+};
+
+__device__ __forceinline__ void warp_logdet(const float* __restrict__ wgt, float* __restrict__ out, int C, int HW, int k, int lane)
+{
+    double s = 0.0;
+    for (int c = lane; c < C; c += 32) s += log(fabs((double)__ldg(wgt + w_index(c, c, k - 1, k - 1, C, k))));
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) out[0] = (float)((double)HW * s);
+}
+
+// value of grad_w at (co, ci, tap) given the correlation sum `s` (grad_w = -s on the mask, 0 outside it)
+__device__ __forceinline__ float finish_grad_w(float s, int co, int ci, int tap, int C, int k, const LogdetFuse& ld)
+{
+    if (tap == 0 && ci > co) return 0.f;
+    float v = -s;
+    if (tap == 0 && ci == co && ld.grad_logdet != nullptr)
+        v += (__ldg(ld.grad_logdet) * (float)ld.HW) / __ldg(ld.w + w_index(co, co, k - 1, k - 1, C, k));
+    return v;
+}
+
 // Upper bound on polls of any device-side wait before it gives up.
 constexpr unsigned kMaxSpins = 1u << 22;
 

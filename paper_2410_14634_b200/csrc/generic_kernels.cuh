@@ -91,7 +91,7 @@ generic_wavefront_kernel(const float* __restrict__ rhs, const float* __restrict_
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(128)
 generic_grad_w_kernel(const float* __restrict__ grad_y, const float* __restrict__ x,
-                      float* __restrict__ grad_w, Geom g)
+                      float* __restrict__ grad_w, Geom g, const LogdetFuse ld)
 {
     const int C = g.C, H = g.H, W = g.W, k = g.k;
     int e = blockIdx.x;
@@ -121,7 +121,7 @@ generic_grad_w_kernel(const float* __restrict__ grad_y, const float* __restrict_
         if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
         __syncthreads();
     }
-    if (threadIdx.x == 0) grad_w[blockIdx.x] = masked_out ? 0.f : -red[0];
+    if (threadIdx.x == 0) grad_w[blockIdx.x] = finish_grad_w(red[0], co, ci, dh * k + dw, C, k, ld);
 }
 
 // ---------------------------------------------------------------------------

@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(32 * (ALLDH ? K * K : TC * K)) gradw_mma_kerne
 // LANES = 1 (one thread per entry, fully coalesced rows) is faster where the entries alone fill the GPU.
 template <int LANES>
 __global__ void __launch_bounds__(256) gradw_reduce_kernel(const float* __restrict__ partials, float* __restrict__ grad_w,
-                                                           int nbc, int C, int K)
+                                                           int nbc, int C, int K, const LogdetFuse ld)
 {
     constexpr int EPW = 32 / LANES;                      // entries per warp
     constexpr int INF = LANES == 1 ? 8 : 16;             // loads in flight per thread
@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(256) gradw_reduce_kernel(const float* __restri
         if (q == 0 && e0 < NA) {
             const int ci = e % C, co = (e / C) % C, tap = e / (C * C);
             const int dh = tap / K, dw = tap % K;
-            grad_w[((co * C + ci) * K + (K - 1 - dh)) * K + (K - 1 - dw)] = (tap == 0 && ci > co) ? 0.f : -s;
+            grad_w[((co * C + ci) * K + (K - 1 - dh)) * K + (K - 1 - dw)] = finish_grad_w(s, co, ci, tap, C, K, ld);
         }
     }
 }
@@ -358,6 +358,7 @@ struct GradWSmallParams {
     int stage;             // floats of dynamic shared memory (the last CTA stages partial sums there)
     int bulk;              // rows are 16-byte aligned multiples of 16 bytes: stage them with bulk copies
     FastDiv div_bands, div_gcpr, div_xcpr, div_rb, div_xr, div_qpr;
+    LogdetFuse ld;         // the log-det's term on the diagonal of grad_w (optional)
 };
 
 template <int C, int K>
@@ -537,7 +538,7 @@ __global__ void __launch_bounds__(GradWSmallShape<C, K>::NT) gradw_small_kernel(
     for (int e = tid; e < NA; e += NT) {
         const int ci_ = e % C, co_ = (e / C) % C, tap = e / (C * C);
         const int dh_ = tap / K, dw_ = tap % K;
-        p.grad_w[((co_ * C + ci_) * K + (K - 1 - dh_)) * K + (K - 1 - dw_)] = (tap == 0 && ci_ > co_) ? 0.f : -red[e];
+        p.grad_w[((co_ * C + ci_) * K + (K - 1 - dh_)) * K + (K - 1 - dw_)] = finish_grad_w(red[e], co_, ci_, tap, C, K, p.ld);
     }
     if (tid == 0) *p.counter = 0u;
 }

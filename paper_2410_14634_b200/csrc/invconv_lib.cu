@@ -219,10 +219,11 @@ int launch_gradw_small_ck(const GradWSmallPlan& gs, const GradWSmallParams& prm,
     return check_launch();
 }
 
-int launch_gradw_small(const GradWSmallPlan& gs, const float* gy, const float* x, float* gw, Geom g, void* ws, cudaStream_t st)
+int launch_gradw_small(const GradWSmallPlan& gs, const float* gy, const float* x, float* gw, Geom g, void* ws, cudaStream_t st,
+                       const LogdetFuse& ld)
 {
     GradWSmallParams prm;
-    prm.gy = gy; prm.x = x; prm.grad_w = gw;
+    prm.gy = gy; prm.x = x; prm.grad_w = gw; prm.ld = ld;
     prm.counter = static_cast<unsigned*>(ws);
     prm.partials = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES);
     prm.B = g.B; prm.H = g.H; prm.W = g.W;
@@ -249,7 +250,8 @@ struct WarpMix {
 };
 
 int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const float* xsaved, float* gw, Geom g,
-                void* ws, cudaStream_t st, const WarpMix* mix = nullptr)
+                void* ws, cudaStream_t st, const WarpMix* mix = nullptr, float* logdet_out = nullptr,
+                const LogdetFuse& ld = LogdetFuse{})
 {
     const WarpPlan pl = plan_warp(g.B, g.C, g.H, g.W, g.k, bwd);
     if (!pl.ok) return INVCONV_UNSUPPORTED;
@@ -261,6 +263,8 @@ int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const fl
     prm.counter = static_cast<unsigned*>(ws);
     prm.partials = ws ? reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES) : nullptr;
     prm.B = g.B; prm.H = g.H; prm.W = g.W; prm.nb = pl.nb; prm.ipc = pl.ipc;
+    prm.logdet_out = bwd ? nullptr : logdet_out;
+    prm.ld = ld;
     if (mix) {
         prm.mix_V = mix->V; prm.mix_s = mix->s; prm.mix_b = mix->b;
         prm.mix_out = bwd ? nullptr : mix->u_out;
@@ -279,7 +283,7 @@ int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const fl
     INVCONV_WARP_CASES(X)
 #undef X
     if (rc || !separate) return rc;
-    return launch_gradw_small(gs, out, xsaved, gw, g, ws, st);
+    return launch_gradw_small(gs, out, xsaved, gw, g, ws, st, ld);
 }
 
 size_t warp_workspace_bytes(int B, int C, int H, int W, int k)
@@ -439,12 +443,12 @@ int launch_gradw_mma_all_inst(const GradWPlan& gp, const GradWParams& prm, cudaS
 }
 
 // grad_w through the tiled correlation kernel; partial sums live behind the transformed kernel in the workspace.
-int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, cudaStream_t st)
+int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, cudaStream_t st, const LogdetFuse& ld)
 {
     const GradWPlan gp = gradw_plan(g.B, g.C, g.H, g.W, g.k);
     const bool aligned = ((reinterpret_cast<uintptr_t>(gy) | reinterpret_cast<uintptr_t>(x)) & 15) == 0;
     if (!gp.ok || !aligned || g.B == 0) {
-        generic_grad_w_kernel<<<g.C * g.C * g.k * g.k, 128, 0, st>>>(gy, x, gw, g);
+        generic_grad_w_kernel<<<g.C * g.C * g.k * g.k, 128, 0, st>>>(gy, x, gw, g, ld);
         return check_launch();
     }
     const size_t na = (size_t)g.k * g.k * g.C * g.C;
@@ -473,10 +477,10 @@ int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, c
     }
     if (rc) return rc;
     if (na < 16384) {       // few entries: four lanes per entry (64 entries per CTA)
-        gradw_reduce_kernel<4><<<(int)((na + 63) / 64), 256, 0, st>>>(prm.partials, gw, shares, g.C, g.k);
+        gradw_reduce_kernel<4><<<(int)((na + 63) / 64), 256, 0, st>>>(prm.partials, gw, shares, g.C, g.k, ld);
     } else {
         const int blocks = (int)((na + 255) / 256 < 4096 ? (na + 255) / 256 : 4096);
-        gradw_reduce_kernel<1><<<blocks, 256, 0, st>>>(prm.partials, gw, shares, g.C, g.k);
+        gradw_reduce_kernel<1><<<blocks, 256, 0, st>>>(prm.partials, gw, shares, g.C, g.k, ld);
     }
     return check_launch();
 }
@@ -534,7 +538,7 @@ int launch_pixel_inst(const TeamPlan& pl, const TeamParams& prm, cudaStream_t st
 }
 
 // Transposed or plain solve through the team family; the transformed kernel goes to the workspace.
-int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, void* ws, cudaStream_t st)
+int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, void* ws, cudaStream_t st, float* logdet_out = nullptr)
 {
     const TeamPlan pl = team_plan(g.B, g.C, g.H, g.W, g.k);
     if (!pl.ok) return INVCONV_UNSUPPORTED;
@@ -544,7 +548,7 @@ int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, 
         auto kern = bwd ? team_solve_kernel<true> : team_solve_kernel<false>;
         const int rc = set_smem_limit(kern, sm);
         if (rc) return rc;
-        kern<<<g.C + (g.C + 31) / 32, 512, sm, st>>>(w, A, g.C, g.k, nullptr, 0, 0u);
+        kern<<<g.C + (g.C + 31) / 32, 512, sm, st>>>(w, A, g.C, g.k, nullptr, 0, 0u, logdet_out, g.H * g.W);
         const int rl = check_launch();
         if (rl) return rl;
     }
@@ -609,32 +613,33 @@ size_t tensor_workspace_bytes(int B, int C, int H, int W, int k)
 
 // grad_w through the tensor-core correlation kernel and the fixed-order reduction over its shares.
 // `partials_offset`: where in the workspace the [shares][k*k][C][C] partial sums go.
-int launch_gradw_tensor(const float* gy, const float* x, float* gw, Geom g, void* ws, size_t partials_offset, cudaStream_t st)
+int launch_gradw_tensor(const float* gy, const float* x, float* gw, Geom g, void* ws, size_t partials_offset, cudaStream_t st,
+                        const LogdetFuse& ld)
 {
     const GradWTensorPlan gt = gradw_tensor_plan(g.B, g.C, g.H, g.W, g.k);
     const bool aligned = ((reinterpret_cast<uintptr_t>(gy) | reinterpret_cast<uintptr_t>(x)) & 15) == 0;
-    if (!gt.ok || !aligned || g.B == 0 || opt(INVCONV_OPT_GRADW_TENSOR_PIPE) == 0) return launch_gradw(gy, x, gw, g, ws, st);
+    if (!gt.ok || !aligned || g.B == 0 || opt(INVCONV_OPT_GRADW_TENSOR_PIPE) == 0) return launch_gradw(gy, x, gw, g, ws, st, ld);
     float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + partials_offset);
     const int rc = invconv_internal::gradw_tensor_launch(gt, gy, x, partials, g, st);
     if (rc) return rc;
     const size_t na = (size_t)g.k * g.k * g.C * g.C;
     if (na < 16384) {
-        gradw_reduce_kernel<4><<<(int)((na + 63) / 64), 256, 0, st>>>(partials, gw, gt.S, g.C, g.k);
+        gradw_reduce_kernel<4><<<(int)((na + 63) / 64), 256, 0, st>>>(partials, gw, gt.S, g.C, g.k, ld);
     } else {
         const int blocks = (int)((na + 255) / 256 < 4096 ? (na + 255) / 256 : 4096);
-        gradw_reduce_kernel<1><<<blocks, 256, 0, st>>>(partials, gw, gt.S, g.C, g.k);
+        gradw_reduce_kernel<1><<<blocks, 256, 0, st>>>(partials, gw, gt.S, g.C, g.k, ld);
     }
     return check_launch();
 }
 
 // Plain or transposed solve on the tensor cores: kernel transform, operand packing, wavefront.
-int launch_tensor(bool bwd, const float* rhs, const float* w, float* out, Geom g, void* ws, cudaStream_t st)
+int launch_tensor(bool bwd, const float* rhs, const float* w, float* out, Geom g, void* ws, cudaStream_t st, float* logdet_out = nullptr)
 {
     const TensorPlan pl = tensor_plan(g.B, g.C, g.H, g.W, g.k);
     if (!pl.ok) return INVCONV_UNSUPPORTED;
     float* A = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES);
     unsigned char* wop = static_cast<unsigned char*>(ws) + tensor_wop_offset(g.B, g.C, g.H, g.W, g.k);
-    return invconv_internal::tensor_launch(pl, bwd, rhs, w, out, g, A, wop, st);
+    return invconv_internal::tensor_launch(pl, bwd, rhs, w, out, g, A, wop, st, logdet_out);
 }
 
 // ---------------------------------------------------------------- dispatch
@@ -660,30 +665,42 @@ size_t workspace_bytes_for(int path, int B, int C, int H, int W, int k)
     return 0;
 }
 
+// `logdet_out` (optional): the layer's log-det, written by the forward kernels themselves where they have a
+// warp to spare (warp family; the kernel transform of the team and tensor families), else by its own launch.
 int launch_forward(int path, const float* y, const float* w, float* x, Geom g,
-                   void* ws, size_t ws_bytes, cudaStream_t st)
+                   void* ws, size_t ws_bytes, cudaStream_t st, float* logdet_out = nullptr)
 {
     (void)ws_bytes;
-    if (g.B == 0) return INVCONV_OK;
-    switch (path) {
-    case INVCONV_PATH_GENERIC:
-        generic_wavefront_kernel<false><<<g.B, 256, 0, st>>>(y, w, x, g);
+    auto separate_logdet = [&]() {
+        if (!logdet_out) return (int)INVCONV_OK;
+        logdet_kernel<<<1, 32, 0, st>>>(w, logdet_out, g.C, g.H, g.W, g.k);
         return check_launch();
+    };
+    if (g.B == 0) return separate_logdet();
+    switch (path) {
+    case INVCONV_PATH_GENERIC: {
+        generic_wavefront_kernel<false><<<g.B, 256, 0, st>>>(y, w, x, g);
+        const int rc = check_launch();
+        return rc ? rc : separate_logdet();
+    }
     case INVCONV_PATH_WARP:
-        return launch_warp(false, y, w, x, nullptr, nullptr, g, ws, st);
+        return launch_warp(false, y, w, x, nullptr, nullptr, g, ws, st, nullptr, logdet_out);
     case INVCONV_PATH_TEAM:
-        return launch_team(false, y, w, x, g, ws, st);
+        return launch_team(false, y, w, x, g, ws, st, logdet_out);
     case INVCONV_PATH_TENSOR:
-        return launch_tensor(false, y, w, x, g, ws, st);
+        return launch_tensor(false, y, w, x, g, ws, st, logdet_out);
     default:
         return INVCONV_UNSUPPORTED;
     }
 }
 
+// `grad_logdet` (optional, one device float): the kernels that write the final grad_w add the log-det's term.
 int launch_backward(int path, const float* gx, const float* x, const float* w, float* gy, float* gw, Geom g,
-                    void* ws, size_t ws_bytes, cudaStream_t st)
+                    void* ws, size_t ws_bytes, cudaStream_t st, const float* grad_logdet = nullptr)
 {
     (void)ws_bytes;
+    LogdetFuse ld;
+    ld.grad_logdet = grad_logdet; ld.w = w; ld.HW = g.H * g.W;
     switch (path) {
     case INVCONV_PATH_GENERIC: {
         if (g.B > 0) {
@@ -692,13 +709,13 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
             if (rc) return rc;
         }
         if (gw) {
-            generic_grad_w_kernel<<<g.C * g.C * g.k * g.k, 128, 0, st>>>(gy, x, gw, g);
+            generic_grad_w_kernel<<<g.C * g.C * g.k * g.k, 128, 0, st>>>(gy, x, gw, g, ld);
             return check_launch();
         }
         return INVCONV_OK;
     }
     case INVCONV_PATH_WARP:
-        return launch_warp(true, gx, w, gy, x, gw, g, ws, st);
+        return launch_warp(true, gx, w, gy, x, gw, g, ws, st, nullptr, nullptr, ld);
     case INVCONV_PATH_TEAM: {
         if (g.B > 0) {
             const int rc = launch_team(true, gx, w, gy, g, ws, st);
@@ -706,7 +723,7 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
         }
         if (gw) {
             const size_t na = sizeof(float) * (size_t)g.k * g.k * g.C * g.C;
-            return launch_gradw_tensor(gy, x, gw, g, ws, INVCONV_WS_CONTROL_BYTES + na + sizeof(float) * (size_t)g.C * g.C, st);
+            return launch_gradw_tensor(gy, x, gw, g, ws, INVCONV_WS_CONTROL_BYTES + na + sizeof(float) * (size_t)g.C * g.C, st, ld);
         }
         return INVCONV_OK;
     }
@@ -715,7 +732,7 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
             const int rc = launch_tensor(true, gx, w, gy, g, ws, st);
             if (rc) return rc;
         }
-        if (gw) return launch_gradw_tensor(gy, x, gw, g, ws, tensor_gradw_offset(g.B, g.C, g.H, g.W, g.k), st);
+        if (gw) return launch_gradw_tensor(gy, x, gw, g, ws, tensor_gradw_offset(g.B, g.C, g.H, g.W, g.k), st, ld);
         return INVCONV_OK;
     }
     default:
@@ -887,19 +904,41 @@ int invconv_forward_logdet(const float* y, const float* w, float* x, float* logd
                            int B, int C, int H, int W, int k, void* stream)
 {
     if (!logdet) return INVCONV_BAD_ARG;
-    const int rc = invconv_forward(y, w, x, B, C, H, W, k, stream);
+    const int rc = check_shape(B, C, H, W, k);
     if (rc) return rc;
-    return invconv_logdet(w, logdet, C, H, W, k, stream);
+    if (!w) return INVCONV_BAD_ARG;
+    if (B > 0 && (!y || !x || y == x)) return INVCONV_BAD_ARG;
+    StreamScratch sc;
+    const int path = resolve_path(B > 0 ? B : 1, C, H, W, k);
+    const size_t need = B > 0 ? workspace_bytes_for(path, B, C, H, W, k) : 0;
+    const int ra = sc.acquire(need, as_stream(stream));
+    if (ra) return ra;
+    return launch_forward(path, y, w, x, Geom{B, C, H, W, k}, sc.p, need, as_stream(stream), logdet);
 }
 
 int invconv_backward_logdet(const float* grad_x, const float* x, const float* w, const float* grad_logdet,
                             float* grad_y, float* grad_w, int B, int C, int H, int W, int k, void* stream)
 {
     if (!grad_logdet || !grad_w) return INVCONV_BAD_ARG;
-    const int rc = invconv_backward(grad_x, x, w, grad_y, grad_w, B, C, H, W, k, stream);
+    const int rc = check_shape(B, C, H, W, k);
     if (rc) return rc;
-    logdet_grad_kernel<<<1, 128, 0, as_stream(stream)>>>(w, grad_logdet, grad_w, C, H, W, k);
-    return check_launch();
+    if (!w) return INVCONV_BAD_ARG;
+    if (B == 0) {
+        // no image: grad_w is the log-det's term alone
+        if (cudaMemsetAsync(grad_w, 0, sizeof(float) * C * C * k * k, as_stream(stream)) != cudaSuccess) {
+            cudaGetLastError();
+            return INVCONV_CUDA_ERROR;
+        }
+        logdet_grad_kernel<<<1, 128, 0, as_stream(stream)>>>(w, grad_logdet, grad_w, C, H, W, k);
+        return check_launch();
+    }
+    if (!grad_x || !x || !grad_y || grad_x == grad_y || x == grad_y) return INVCONV_BAD_ARG;
+    StreamScratch sc;
+    const int path = resolve_path(B, C, H, W, k);
+    const size_t need = workspace_bytes_for(path, B, C, H, W, k);
+    const int ra = sc.acquire(need, as_stream(stream));
+    if (ra) return ra;
+    return launch_backward(path, grad_x, x, w, grad_y, grad_w, Geom{B, C, H, W, k}, sc.p, need, as_stream(stream), grad_logdet);
 }
 
 size_t invconv_step_scratch_bytes(int B, int C, int H, int W, int k)

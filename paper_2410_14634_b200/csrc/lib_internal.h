@@ -38,7 +38,7 @@ int warp_step_backward(const float* grad_u, const float* x, const float* w, cons
 
 // tensor_lib.cu: the tcgen05 wavefront (kernel transform into A, operand packing into wop, solve).
 int tensor_launch(const invconv::TensorPlan& pl, bool bwd, const float* rhs, const float* w, float* out,
-                  invconv::Geom g, float* A, unsigned char* wop, cudaStream_t st);
+                  invconv::Geom g, float* A, unsigned char* wop, cudaStream_t st, float* logdet_out = nullptr);
 int tensor_read_clear_status(int* status_out);
 
 // tensor_lib.cu: the tcgen05 correlation kernel of grad_w; partial sums [pl.S][k*k][C][C] go to `partials`.

@@ -52,10 +52,13 @@ namespace cg = cooperative_groups;
 // ---------------------------------------------------------------------------
 template <bool BWD>
 __global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K,
-                                                         unsigned char* __restrict__ wop, int NCH, unsigned wbytes)
+                                                         unsigned char* __restrict__ wop, int NCH, unsigned wbytes,
+                                                         float* __restrict__ logdet_out, int HW)
 {
     extern __shared__ __align__(128) float sm[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the wavefront kernel may set itself up meanwhile
+    if (logdet_out != nullptr && blockIdx.x == gridDim.x - 1 && threadIdx.x >= 480)
+        warp_logdet(w, logdet_out, C, HW, K, threadIdx.x & 31);        // the layer's log-det, by a warp of the lightest CTA
     const int KK = K * K, ctr = KK - 1;
     const int tid = threadIdx.x, NT = blockDim.x;
     const int b = blockIdx.x;

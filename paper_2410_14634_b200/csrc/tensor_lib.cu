@@ -49,7 +49,7 @@ int launch_tensor_inst(const TensorPlan& pl, const TensorParams& prm, cudaStream
 namespace invconv_internal {
 
 int tensor_launch(const TensorPlan& pl, bool bwd, const float* rhs, const float* w, float* out, Geom g,
-                  float* A, unsigned char* wop, cudaStream_t st)
+                  float* A, unsigned char* wop, cudaStream_t st, float* logdet_out)
 {
     if (((reinterpret_cast<uintptr_t>(rhs) | reinterpret_cast<uintptr_t>(out)) & 15) != 0) return INVCONV_UNSUPPORTED;
     {
@@ -57,7 +57,7 @@ int tensor_launch(const TensorPlan& pl, bool bwd, const float* rhs, const float*
         auto kern = bwd ? team_solve_kernel<true> : team_solve_kernel<false>;
         const int rc = set_smem_limit(kern, sm);
         if (rc) return rc;
-        kern<<<g.C + (g.C + 31) / 32, 512, sm, st>>>(w, A, g.C, g.k, wop, pl.NCH, pl.wbytes);
+        kern<<<g.C + (g.C + 31) / 32, 512, sm, st>>>(w, A, g.C, g.k, wop, pl.NCH, pl.wbytes, logdet_out, g.H * g.W);
         const int rl = check_launch();
         if (rl) return rl;
     }

@@ -70,6 +70,8 @@ struct WarpParams {
     const float* mix_b = nullptr;   // [C] (forward only)
     float* mix_out = nullptr;       // forward: u [B][C][H][W], written beside x
     int mix_in = 0;                 // backward: rhs holds grad_u; grad_x = s * (V^T grad_u) is formed after the load
+    float* logdet_out = nullptr;    // forward: CTA 0 also writes the layer's log-det (one float)
+    LogdetFuse ld;                  // backward: the log-det's term on the diagonal of grad_w
 };
 
 template <int C> struct ColVec;
@@ -888,6 +890,10 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
         }
     }
     if (threadIdx.x < p.ipc * p.nb) progress[threadIdx.x] = 0;
+    if constexpr (!BWD) {
+        // the log-det rides in the shadow of the image's arrival: one warp of one CTA, C double-precision logarithms
+        if (p.logdet_out != nullptr && blockIdx.x == 0 && warp == 0) warp_logdet(p.w, p.logdet_out, C, HW, K, lane);
+    }
     build_transformed_kernel<C, K, BWD>(p.w, As);
     __syncthreads();
     WARP_TT(1);
@@ -1044,8 +1050,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
                     else for (int b = 0; b < G; ++b) s += __ldcg(p.partials + (size_t)b * S::NA + i);
                     const int ci = i % C, co = (i / C) % C, tap = i / (C * C);
                     const int dh = tap / K, dw = tap % K;
-                    const bool masked_out = (tap == 0 && ci > co);
-                    p.grad_w[((co * C + ci) * K + (K - 1 - dh)) * K + (K - 1 - dw)] = masked_out ? 0.f : -s;
+                    p.grad_w[((co * C + ci) * K + (K - 1 - dh)) * K + (K - 1 - dw)] = finish_grad_w(s, co, ci, tap, C, K, p.ld);
                 }
                 if (threadIdx.x == 0) *p.counter = 0u;
             }

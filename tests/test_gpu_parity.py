@@ -209,11 +209,14 @@ def test_masked_conv_matches_oracle(B, oracle, shape, path):
     assert nmax_err(y.cpu().numpy(), oracle.masked_conv(x, w)) <= 1e-5
 
 
-@pytest.mark.parametrize("shape", [(4, 3, 16, 16, 3), (3, 1, 28, 28, 3), (2, 12, 8, 8, 3), (2, 5, 6, 7, 2)],
+@pytest.mark.parametrize("shape", [(4, 3, 16, 16, 3), (3, 1, 28, 28, 3), (2, 12, 8, 8, 3), (2, 5, 6, 7, 2),
+                                   (2, 3, 64, 64, 5), (1, 1, 250, 257, 3), (9, 48, 16, 16, 3), (3, 96, 8, 8, 3), (1, 3, 8, 8, 7)],
                          ids=lambda s: "x".join(map(str, s)))
 def test_training_step_calls_with_the_log_det_folded_in(B, oracle, shape):
     """invconv_forward_logdet / invconv_backward_logdet against the oracle's x, logdet, grad_y and
-    grad_w + grad_logdet * d logdet / d w."""
+    grad_w + grad_logdet * d logdet / d w, for every place the log-det is emitted from (the warp kernel, the
+    separate grad_w kernel of large images, the kernel transform and grad_w reductions of the team and tensor
+    families, the fallback kernels)."""
     import torch
     Bn, C, H, W, k = shape
     w, y, gx = workloads.make_custom(500 + sum(shape), Bn, C, H, W, k, sigma=0.05 / np.sqrt(C))
