@@ -66,9 +66,10 @@ enum invconv_path {
  * substitution over the H+W-1 anti-diagonals (Section 3, Eq. 1 solved for
  * x_q; Supplementary "Input Padding and Kernel Masking").
  *   y [B,C,H,W] in, w [C,C,k,k] in, x [B,C,H,W] out.
- * Uses stream-ordered scratch from the device's default memory pool when the
- * shape needs a workspace (see invconv_workspace_bytes); use the _ws form to
- * supply the scratch yourself. */
+ * Uses stream-ordered scratch when the shape needs a workspace (see
+ * invconv_workspace_bytes), taken from a memory pool the library creates per
+ * device on first use and keeps (freed blocks stay cached in it); use the _ws
+ * form to supply the scratch yourself. */
 int invconv_forward(const float* y, const float* w, float* x,
                     int B, int C, int H, int W, int k, void* stream);
 
@@ -140,7 +141,7 @@ int invconv_backward_logdet(const float* grad_x, const float* x, const float* w,
  * For shapes of the warp-shuffle family whose images fit shared memory the neighbours are applied inside the
  * wavefront kernel (u is written while x is stored; the incoming gradient is transformed as it is loaded);
  * other shapes run the layer's kernels and per-pixel kernels one after the other -- same results.  Scratch
- * comes from the device's stream-ordered memory pool.  Argument rules and errors as for invconv_forward. */
+ * comes from the library's stream-ordered memory pool.  Argument rules and errors as for invconv_forward. */
 int invconv_flow_step_forward(const float* y, const float* w, const float* s, const float* b, const float* V,
                               float* x, float* u, float* logdet, int B, int C, int H, int W, int k, void* stream);
 int invconv_flow_step_backward(const float* grad_u, const float* x, const float* w, const float* s, const float* b,
@@ -194,7 +195,7 @@ int invconv_step_host(const float* y_host, const float* w_host, const float* gra
  * runs inside another framework's callback -- and from then on may call
  * neither cudaMalloc nor a pooled allocator.  The other backward entry points
  * need scratch memory (a completion counter and per-CTA partial sums of
- * grad_w) that either the library takes from the device's memory pool
+ * grad_w) that either the library takes from its stream-ordered memory pool
  * (invconv_backward) or the caller provides (invconv_backward_ws).  This
  * variant keeps that scratch in a fixed array of INVCONV_NOALLOC_SCRATCH_BYTES
  * that is part of the library image itself: every GPU that loads the library

@@ -189,7 +189,7 @@ struct Scratch {
     {
         st = s;
         if (bytes == 0) return INVCONV_OK;
-        if (cudaMallocAsync(&p, bytes, st) != cudaSuccess) { cudaGetLastError(); p = nullptr; return INVCONV_CUDA_ERROR; }
+        { const int rc = invconv_internal::scratch_alloc(&p, bytes, st); if (rc) { p = nullptr; return rc; } }
         if (cudaMemsetAsync(p, 0, INVCONV_WS_CONTROL_BYTES, st) != cudaSuccess) { cudaGetLastError(); return INVCONV_CUDA_ERROR; }
         return INVCONV_OK;
     }

@@ -366,6 +366,34 @@ int launch_masked_conv_small(const float* x, const float* w, float* y, Geom g, c
 // ---------------------------------------------------------------- team family
 }  // namespace
 namespace invconv_internal {
+// Scratch comes from a memory pool the library owns (one per device, created on first use) whose release
+// threshold is unlimited: memory freed with cudaFreeAsync stays in the pool across synchronisations, so the
+// steady state allocates nothing from the driver (the default pool would hand its memory back at every
+// synchronisation and pay for a fresh allocation, about 200 us, on the next call).
+int scratch_alloc(void** out, size_t bytes, cudaStream_t st)
+{
+    static std::mutex mu;
+    static cudaMemPool_t pools[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return INVCONV_CUDA_ERROR; }
+    cudaMemPool_t pool;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!pools[dev]) {
+            cudaMemPoolProps props = {};
+            props.allocType = cudaMemAllocationTypePinned;
+            props.location.type = cudaMemLocationTypeDevice;
+            props.location.id = dev;
+            if (cudaMemPoolCreate(&pools[dev], &props) != cudaSuccess) { cudaGetLastError(); pools[dev] = nullptr; return INVCONV_CUDA_ERROR; }
+            unsigned long long keep = ~0ull;
+            cudaMemPoolSetAttribute(pools[dev], cudaMemPoolAttrReleaseThreshold, &keep);
+        }
+        pool = pools[dev];
+    }
+    if (cudaMallocFromPoolAsync(out, bytes, pool, st) != cudaSuccess) { cudaGetLastError(); *out = nullptr; return INVCONV_CUDA_ERROR; }
+    return INVCONV_OK;
+}
+
 int sm_count()
 {
     static std::atomic<int> cached[64];
@@ -740,14 +768,15 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
     }
 }
 
-// Stream-ordered scratch for the entry points that take no workspace.
+// Stream-ordered scratch for the entry points that take no workspace (see invconv_internal::scratch_alloc).
 struct StreamScratch {
     void* p = nullptr;
     cudaStream_t st;
     int acquire(size_t bytes, cudaStream_t s) {
         st = s;
         if (bytes == 0) return INVCONV_OK;
-        if (cudaMallocAsync(&p, bytes, st) != cudaSuccess) { cudaGetLastError(); p = nullptr; return INVCONV_CUDA_ERROR; }
+        const int rc = invconv_internal::scratch_alloc(&p, bytes, st);
+        if (rc) { p = nullptr; return rc; }
         if (cudaMemsetAsync(p, 0, INVCONV_WS_CONTROL_BYTES, st) != cudaSuccess) { cudaGetLastError(); return INVCONV_CUDA_ERROR; }
         return INVCONV_OK;
     }
@@ -882,6 +911,14 @@ int masked_conv_forward(const float* x, const float* w, float* y, int B, int C, 
     if (g_forced_path.load() != INVCONV_PATH_GENERIC) {
         const int rs = launch_masked_conv_small(x, w, y, Geom{B, C, H, W, k}, as_stream(stream));
         if (rs != INVCONV_UNSUPPORTED) return rs;
+        // many channels: the tensor cores (forcing the team family keeps the FMA tile kernel, for comparison)
+        const ConvTensorPlan ct = plan_conv_tensor(B, C, H, W, k, kMaxDynSmem, sm_count());
+        if (ct.ok && g_forced_path.load() != INVCONV_PATH_TEAM) {
+            StreamScratch sc;
+            const int ra = sc.acquire(ct.pack_bytes, as_stream(stream));
+            if (ra) return ra;
+            return invconv_internal::conv_tensor_launch(ct, x, w, y, Geom{B, C, H, W, k}, static_cast<unsigned char*>(sc.p), as_stream(stream));
+        }
         const int rt = launch_masked_conv_tile(x, w, y, Geom{B, C, H, W, k}, as_stream(stream));
         if (rt != INVCONV_UNSUPPORTED) return rt;
     }

@@ -15,6 +15,9 @@ constexpr size_t kMaxDynSmem = 226 * 1024;   // 227 KiB per CTA minus the kernel
 // Counts the launch and turns cudaGetLastError into a status code.
 int check_launch();
 
+// Stream-ordered device scratch from the library's own memory pool; release with cudaFreeAsync on the same stream.
+int scratch_alloc(void** out, size_t bytes, cudaStream_t st);
+
 // Multiprocessors of the current device (cached per device).
 int sm_count();
 
@@ -40,6 +43,10 @@ int warp_step_backward(const float* grad_u, const float* x, const float* w, cons
 int tensor_launch(const invconv::TensorPlan& pl, bool bwd, const float* rhs, const float* w, float* out,
                   invconv::Geom g, float* A, unsigned char* wop, cudaStream_t st, float* logdet_out = nullptr);
 int tensor_read_clear_status(int* status_out);
+
+// tensor_lib.cu: y = f(x) on the tensor cores; `pack` is device scratch of pl.pack_bytes bytes.
+int conv_tensor_launch(const invconv::ConvTensorPlan& pl, const float* x, const float* w, float* y, invconv::Geom g,
+                       unsigned char* pack, cudaStream_t st);
 
 // tensor_lib.cu: the tcgen05 correlation kernel of grad_w; partial sums [pl.S][k*k][C][C] go to `partials`.
 int gradw_tensor_launch(const invconv::GradWTensorPlan& pl, const float* gy, const float* x, float* partials,

@@ -11,6 +11,7 @@
 #include "team_kernels.cuh"      // team_solve_kernel: the kernel transform L^-1 W_delta
 #include "tensor_kernels.cuh"
 #include "gradw_tensor.cuh"
+#include "conv_tensor.cuh"
 
 using namespace invconv;
 
@@ -98,6 +99,39 @@ int gradw_tensor_launch(const GradWTensorPlan& pl, const float* gy, const float*
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
     if (e != cudaSuccess) {
         std::fprintf(stderr, "invconv: grad_w tensor launch failed: %s\n", cudaGetErrorString(e));
+        cudaGetLastError();
+        return INVCONV_CUDA_ERROR;
+    }
+    return check_launch();
+}
+
+int conv_tensor_launch(const ConvTensorPlan& pl, const float* x, const float* w, float* y, Geom g, unsigned char* pack, cudaStream_t st)
+{
+    const int total = g.k * g.k * (g.C / 8) * g.C;
+    conv_pack_kernel<<<(total + 255) / 256, 256, 0, st>>>(w, pack, g.C, g.k);
+    int rc = check_launch();
+    if (rc) return rc;
+    auto kern = conv_tensor_kernel;
+    rc = set_smem_limit(kern, pl.smem);
+    if (rc) return rc;
+    ConvTensorParams prm;
+    prm.x = x; prm.pack = pack; prm.y = y;
+    prm.B = g.B; prm.C = g.C; prm.H = g.H; prm.W = g.W; prm.K = g.k;
+    prm.RB = pl.RB; prm.Wp = pl.Wp; prm.nbands = pl.nbands; prm.ntiles = pl.ntiles; prm.slots = pl.slots; prm.spi = pl.spi;
+    prm.tmem_cols = pl.tmem_cols; prm.x_bytes = pl.x_bytes; prm.wstage_bytes = pl.wstage_bytes;
+    prm.off_w = pl.off_w; prm.off_bar = pl.off_bar;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(pl.grid);
+    cfg.blockDim = dim3(kConvTensorThreads);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // x is staged while the kernel is being packed
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
+    if (e != cudaSuccess) {
+        std::fprintf(stderr, "invconv: tensor convolution launch failed: %s\n", cudaGetErrorString(e));
         cudaGetLastError();
         return INVCONV_CUDA_ERROR;
     }

@@ -95,4 +95,50 @@ inline GradWTensorPlan plan_gradw_tensor(int B, int C, int H, int W, int K, size
     return pl;
 }
 
+// Masked convolution y = f(x) on the tensor cores (conv_tensor.cuh): lanes are the padded pixel slots of a band of
+// rows of one image, taps are row offsets of the staged x operand, weights stream through a ring of stages.
+struct ConvTensorPlan {
+    bool ok = false;
+    int RB = 0, Wp = 0, nbands = 0, ntiles = 0, grid = 0, slots = 0;
+    int spi = 0;                    // weight stages per issuing warp (ring depth)
+    unsigned tmem_cols = 0, x_bytes = 0, wstage_bytes = 0, off_w = 0, off_bar = 0;
+    size_t smem = 0, pack_bytes = 0;
+};
+
+constexpr int kConvTensorThreads = 352;       // warps 0-7 stage x (0-3 also write y); warps 8, 9 issue MMAs; warp 10 loads weights
+constexpr int kConvTensorMaxSpi = 4;            // at most 4 weight stages per issuing warp
+
+inline ConvTensorPlan plan_conv_tensor(int B, int C, int H, int W, int K, size_t max_smem, int sms)
+{
+    ConvTensorPlan pl;
+    if (C % 16 != 0 || C < 16 || C > 64 || K < 2 || K > 5 || B < 1) return pl;
+    pl.Wp = W + K - 1;
+    if (pl.Wp > 128) return pl;
+    pl.wstage_bytes = (unsigned)((C / 8) * 4 * C * 16);
+    for (pl.RB = 128 / pl.Wp < H ? 128 / pl.Wp : H; pl.RB >= 1; --pl.RB) {
+        pl.slots = (K - 1) + (K - 1) * pl.Wp + 128 + pl.Wp;                 // every tap's 128 rows stay inside the buffer
+        const int need = (K - 1) + (pl.RB + K - 1) * pl.Wp;
+        if (need > pl.slots) pl.slots = need;
+        pl.x_bytes = (unsigned)(((size_t)(C / 8) * 4 * pl.slots * 16 + 127) & ~(size_t)127);
+        pl.off_w = pl.x_bytes;
+        // as many weight stages as fit (the bytes in flight from L2 set the streaming rate), at least two per warp
+        for (pl.spi = kConvTensorMaxSpi; pl.spi >= 2; --pl.spi) {
+            pl.off_bar = pl.off_w + 2 * pl.spi * pl.wstage_bytes;
+            pl.smem = (size_t)pl.off_bar + 256;
+            if (pl.smem <= max_smem) break;
+        }
+        if (pl.spi >= 2) break;
+    }
+    if (pl.RB < 1) return pl;
+    pl.nbands = (H + pl.RB - 1) / pl.RB;
+    pl.ntiles = B * pl.nbands;
+    pl.grid = pl.ntiles < sms ? pl.ntiles : sms;
+    unsigned cols = 32;
+    while (cols < (unsigned)(2 * C)) cols *= 2;
+    pl.tmem_cols = cols;
+    pl.pack_bytes = (size_t)K * K * pl.wstage_bytes;
+    pl.ok = true;
+    return pl;
+}
+
 }  // namespace invconv

@@ -187,9 +187,14 @@ def test_paper_setting_unit_diagonal_one_channel(B, oracle, path):
     assert float(B.invconv_logdet(dev(w), 12, 10).item()) == 0.0
 
 
-@pytest.mark.parametrize("path", ["auto", "generic"])
+@pytest.mark.parametrize("path", ["auto", "generic", "team"])
 @pytest.mark.parametrize("shape", [(3, 1, 28, 28, 3), (2, 3, 32, 32, 3), (2, 3, 40, 45, 5), (1, 2, 7, 70, 2), (2, 4, 9, 9, 5),
-                                   (2, 12, 16, 16, 3), (1, 48, 8, 8, 3), (1, 3, 5, 5, 7),
+                                   # tensor-core kernel ("auto" at C = 16..64; "team" keeps the FMA tile kernel): every k
+                                   # it serves, bands that do not fill the lanes, ragged last band, wide and 1-pixel-high
+                                   # images, more tiles than CTAs, the two 48-channel benchmark shapes
+                                   (3, 16, 16, 16, 3), (2, 32, 9, 20, 5), (1, 48, 8, 8, 3), (2, 64, 12, 7, 4), (3, 16, 1, 100, 2),
+                                   (170, 16, 4, 4, 3), (1, 48, 50, 30, 5), (64, 48, 16, 16, 5), (64, 48, 16, 16, 3),
+                                   (2, 12, 16, 16, 3), (1, 3, 5, 5, 7),
                                    # many channels (register-tiled kernel): ragged widths, several bands per image,
                                    # several images per CTA, channel counts off the tile sizes, every k it serves
                                    (3, 5, 7, 9, 2), (2, 13, 20, 20, 4), (1, 33, 6, 10, 5), (1, 6, 40, 36, 3), (2, 7, 5, 5, 1),
