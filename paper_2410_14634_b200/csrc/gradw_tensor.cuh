@@ -14,7 +14,6 @@
 // adds them in a fixed order.
 #pragma once
 
-#include <cstdio>
 
 #include "common.cuh"
 #include "tma.cuh"
@@ -77,10 +76,6 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
         }
     };
 
-#ifdef INVCONV_TENSOR_TIMING
-    const long long tk0_ = clock64();
-    long long tw_ = 0, tl_ = 0, ts_ = 0;
-#endif
     int my_units = 0;
     for (int u = share; u < nunits; u += p.S) ++my_units;
 
@@ -101,17 +96,12 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
             left[j] = q > 0;
         }
         const size_t copy_bytes = (size_t)nchunk * planeC;
+        const bool shuffle_left = (32 % QW) == 0;          // a row's quads never straddle a warp
         int it = 0;
         for (int u = share; u < nunits; u += p.S, ++it) {
             const int n = u / p.nbands, r = u - n * p.nbands;
             const int st = it & 1;
-#ifdef INVCONV_TENSOR_TIMING
-            long long tt0_ = clock64();
-#endif
             if (it >= 2) wait_bar(empty + st, ((it >> 1) - 1) & 1);
-#ifdef INVCONV_TENSOR_TIMING
-            tw_ += clock64() - tt0_; tt0_ = clock64();
-#endif
             unsigned char* sa = gsmem + (size_t)st * p.stage_bytes;
             unsigned char* sb = sa + copy_bytes;
             const float* gyb = p.gy + (size_t)n * C * HW + (size_t)r * RB * W;        // first row of the band
@@ -129,8 +119,18 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
                         a[j] = __ldg(reinterpret_cast<const float4*>(gyb + goff[j0 + j]));
                         if (h >= dh) {
                             b1[j] = __ldg(reinterpret_cast<const float4*>(xb + goff[j0 + j]));
-                            if (left[j0 + j]) b0[j] = __ldg(reinterpret_cast<const float4*>(xb + goff[j0 + j] - 4));
+                            if (left[j0 + j] && !shuffle_left) b0[j] = __ldg(reinterpret_cast<const float4*>(xb + goff[j0 + j] - 4));
                         }
+                    }
+                }
+                if (shuffle_left) {
+                    // the quad to the left is the previous lane's quad (quads of a row are consecutive lanes)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        float4 t;
+                        t.x = __shfl_up_sync(0xffffffffu, b1[j].x, 1); t.y = __shfl_up_sync(0xffffffffu, b1[j].y, 1);
+                        t.z = __shfl_up_sync(0xffffffffu, b1[j].z, 1); t.w = __shfl_up_sync(0xffffffffu, b1[j].w, 1);
+                        if (left[j0 + j]) b0[j] = t;
                     }
                 }
 #pragma unroll
@@ -149,18 +149,9 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
                     if (K > 4) *reinterpret_cast<float4*>(db_ + 4 * copy_bytes) = make_float4(x0, x1, x2, x3);
                 }
             }
-#ifdef INVCONV_TENSOR_TIMING
-            tl_ += clock64() - tt0_; tt0_ = clock64();
-#endif
             fence_proxy_async();
             mbar_arrive(full + st);
-#ifdef INVCONV_TENSOR_TIMING
-            ts_ += clock64() - tt0_;
-#endif
         }
-#ifdef INVCONV_TENSOR_TIMING
-        if (tid == 0 && blockIdx.x == 0) printf("gradw producer: units %d total %lld | wait-empty %lld stage %lld fence+arrive %lld\n", my_units, clock64() - tk0_, tw_, tl_, ts_);
-#endif
         // ------------------------------------------------ accumulators -> partial sums (lane = co)
         if (warp < 4) {
             wait_bar(done, 0);
@@ -205,9 +196,6 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
             umma::commit(empty + st);
         }
         umma::commit(done);
-#ifdef INVCONV_TENSOR_TIMING
-        if (dw == 0 && blockIdx.x == 0) printf("gradw issuer0: total %lld\n", clock64() - tk0_);
-#endif
     }
     umma::fence_before_sync();
     __syncthreads();

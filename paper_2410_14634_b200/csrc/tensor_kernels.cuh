@@ -32,7 +32,6 @@
 #pragma once
 
 #include <cuda_bf16.h>
-#include <cstdio>
 
 #include "common.cuh"
 #include "tma.cuh"
@@ -66,11 +65,6 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b)
 // ---------------------------------------------------------------------------
 namespace tensor_detail {
 
-#ifdef INVCONV_TENSOR_TIMING
-#define TENSOR_TT(i) do { if (timing_) { const long long now_ = clock64(); tacc_[i] += now_ - tlast_; tlast_ = now_; } } while (0)
-#else
-#define TENSOR_TT(i) do { } while (0)
-#endif
 
 constexpr long long kWaitLimit = 1ll << 24;      // SM cycles (about 8 ms) before a wait gives up
 
@@ -201,21 +195,14 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
         const uint32_t own_col = rank * CS + wg * 4;
         unsigned nd = 0;            // diagonals processed so far (all groups): buffer = nd & 1, phase = (nd >> 1) & 1
         unsigned ng = 0;            // groups processed so far
-#ifdef INVCONV_TENSOR_TIMING
-        const bool timing_ = tid == 65 && blockIdx.x == 0;
-        long long tacc_[11] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, tlast_ = clock64();
-        const long long tstart_ = tlast_;
-#endif
         for (int g = cluster_id; g < p.ngroups; g += p.ncl, ++ng) {
             const int img = g * I + i;
             const bool img_ok = img < p.B;
             wait_bar(ybar, ng & 1, gave_up);
-            TENSOR_TT(0);
             int slot_d = 0;
             for (int d = 0; d < D; ++d, ++nd) {
                 const unsigned b = nd & 1, ph = (nd >> 1) & 1;
                 wait_bar(accbar, nd & 1, gave_up);
-                TENSOR_TT(1);
                 umma::fence_after_sync();
                 uint32_t acc[CG][8], own[4];
                 const uint32_t col = (uint32_t)(slot_d * C);
@@ -227,7 +214,6 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
                 for (int q = 0; q < CG; ++q) umma::tmem_ld_fence(acc[q]);
                 umma::tmem_ld_fence(own);
                 umma::fence_before_sync();
-                TENSOR_TT(2);
                 // partial sums of the other CTAs' output channels go to their owners
                 const uint32_t boff = b * recv_buf_floats * 4, bbar = b * 8;
                 const int w = d - h;
@@ -241,9 +227,7 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
                                                                                   __uint_as_float(acc[q][6]), __uint_as_float(acc[q][7])), remote_bar[q] + bbar);
                     }
                 }
-                TENSOR_TT(3);
                 wait_bar(rbar + b, ph, gave_up);
-                TENSOR_TT(4);
                 if (tid == 0) mbar_expect_tx(rbar + b, recv_bytes((d + 2) % D));   // arm the phase two diagonals ahead
                 // own channels 4wg .. 4wg+3: sum over the CTAs in rank order
                 const float* recv_b = s_recv + b * recv_buf_floats + wg * 128 * 4 + m * 4;
@@ -251,7 +235,6 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
 #pragma unroll
                 for (int sl = 0; sl < R - 1; ++sl)
                     pa[sl] = on_diag ? *reinterpret_cast<const float4*>(recv_b + (size_t)sl * 128 * CS) : make_float4(0.f, 0.f, 0.f, 0.f);
-                TENSOR_TT(10);
                 float v[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int pr = 0; pr < R; ++pr) {
@@ -270,7 +253,6 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
 #pragma unroll
                     for (int j = 0; j < 4; ++j) v[j] = 0.f;
                 }
-                TENSOR_TT(5);
                 {   // this warpgroup's half of the operand row: tf32 plane wg, 8 bytes of each bf16 plane
                     unsigned char* xb = s_x + b * xbuf_bytes;
                     const int row = HALO + m;
@@ -283,36 +265,22 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
                     *reinterpret_cast<uint2*>(xb + ((size_t)3 * ROWS + row) * 16 + wg * 8) =
                         make_uint2(pack_bf16x2(v[0] - hi[0], v[1] - hi[1]), pack_bf16x2(v[2] - hi[2], v[3] - hi[3]));
                 }
-                TENSOR_TT(6);
                 fence_proxy_async();
-                TENSOR_TT(7);
                 mbar_arrive(xfull + b);
-                TENSOR_TT(8);
                 if (valid) {
                     const int hh = p.rot ? H - 1 - h : h, ww = p.rot ? W - 1 - w : w;
                     float* dst = s_stage + (size_t)i * p.stage_img + (size_t)(wg * 4) * H * W + (size_t)hh * W + ww;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) dst[(size_t)j * H * W] = v[j];
                 }
-                TENSOR_TT(9);
             }
             fence_proxy_async();          // the staged slice is stored by bulk copies
             mbar_arrive(xdone);
         }
-#ifdef INVCONV_TENSOR_TIMING
-        if (timing_) printf("tensor epi: total %lld | ywait %lld accwait %lld tmemld %lld send %lld rwait %lld ldrecv %lld sum %lld opstore %lld fence %lld arrive %lld staging %lld\n",
-                            clock64() - tstart_, tacc_[0], tacc_[1], tacc_[2], tacc_[3], tacc_[4], tacc_[10], tacc_[5], tacc_[6], tacc_[7], tacc_[8], tacc_[9]);
-#endif
     } else if (warp == 8) {
         // ------------------------------------------------ MMA issue (one thread)
         if (tid == 256) {
-#ifdef INVCONV_TENSOR_TIMING
-            const bool timing_ = blockIdx.x == 0;
-            long long tacc_[8] = {0, 0, 0, 0, 0, 0, 0, 0}, tlast_ = clock64();
-            const long long tstart_ = tlast_;
-#endif
             wait_bar(wbar, 0, gave_up);
-            TENSOR_TT(0);
             const unsigned xplane = ROWS * 16;
             constexpr unsigned wplane = KC * 16;
             // descriptors of row 0 (no lane shift) of buffer 0 / of tap row 0 of dh = 0; everything else is an offset in 16-byte units
@@ -365,12 +333,10 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
             for (int g = cluster_id; g < p.ngroups; g += p.ncl) {
                 for (int t = 0; t < S && t < D; ++t) rhs_tap(t);
                 umma::commit(accbar);
-                TENSOR_TT(1);
                 int slot_d = 0;
                 for (int d = 0; d < D; ++d, ++nd) {
                     const unsigned b = nd & 1;
                     wait_bar(xfull + b, (nd >> 1) & 1, gave_up);
-                    TENSOR_TT(2);
                     umma::fence_after_sync();
                     if (d + 1 < D) {       // taps (0,1) and (1,0): the next diagonal waits for these only
                         const uint32_t dcol = tmem + (uint32_t)((slot_d + 1 == S ? 0 : slot_d + 1) * C);
@@ -381,21 +347,14 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
                         umma::mma_bf16(dcol, xd_bf + xo - (uint64_t)I, w10_bf, idesc_bf | cbits, 1u);
                         umma::commit(accbar);
                     }
-                    TENSOR_TT(3);
                     if (d + S < D) rhs_tap(slot_d);
-                    TENSOR_TT(4);
                     if (K > 2) window(b, d, slot_d, 0, 2, K - 2);
                     window(b, d, slot_d, 1, 1, K - 1);
 #pragma unroll
                     for (int dh = 2; dh < K; ++dh) window(b, d, slot_d, dh, 0, K);
                     slot_d = slot_d + 1 == S ? 0 : slot_d + 1;
-                    TENSOR_TT(5);
                 }
             }
-#ifdef INVCONV_TENSOR_TIMING
-            if (timing_) printf("tensor mma: total %lld | wwait %lld prologue %lld xwait %lld crit %lld rhs %lld rest %lld\n",
-                                clock64() - tstart_, tacc_[0], tacc_[1], tacc_[2], tacc_[3], tacc_[4], tacc_[5]);
-#endif
         }
         __syncwarp();
     } else {

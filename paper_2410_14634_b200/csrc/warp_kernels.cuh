@@ -866,12 +866,6 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     // let the next kernel on the stream be scheduled now; it waits at its own griddepcontrol.wait until this
     // kernel has completed, so only its launch latency overlaps
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-#ifdef INVCONV_WARP_TIMING
-    long long tw_[6]; tw_[0] = clock64();
-#define WARP_TT(i) tw_[i] = clock64()
-#else
-#define WARP_TT(i) do { } while (0)
-#endif
     // the image's bulk copy goes out first; the kernel transform below overlaps its latency
     if (!GLB && leader && p.bulk) {
         mbar_init(&bars[li], 1);
@@ -896,7 +890,6 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     }
     build_transformed_kernel<C, K, BWD>(p.w, As);
     __syncthreads();
-    WARP_TT(1);
 
     bool ok = true;
     if (has_img) {
@@ -931,7 +924,6 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
         }
     }
     if (has_img) {
-        WARP_TT(2);
         if (ok) {
             if constexpr (CS)
                 ok = wavefront_block_cs<C, K, MULTI>(img, As, H, W, BWD ? HW - 1 : 0, BWD ? -1 : 1, j, progress + li * p.nb,
@@ -949,7 +941,6 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
         }
         if (!ok && lane == 0) raise_status(INVCONV_TIMEOUT);
     }
-    WARP_TT(3);
     __syncthreads();
 
     if (!GLB && has_img) {
@@ -1056,14 +1047,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
             }
         }
     }
-    WARP_TT(4);
     if (!GLB && p.bulk && leader && CHW * 4 > 16384) bulk_wait_read0();
-#ifdef INVCONV_WARP_TIMING
-    WARP_TT(5);
-    if (threadIdx.x == 0 && blockIdx.x == 0)
-        printf("warp timing (cycles): setup %lld | load wait %lld | wavefront %lld | store+gradw %lld | store drain %lld\n",
-               tw_[1] - tw_[0], tw_[2] - tw_[1], tw_[3] - tw_[2], tw_[4] - tw_[3], tw_[5] - tw_[4]);
-#endif
 }
 
 // Dynamic shared memory the kernel needs for a launch shape.
