@@ -380,6 +380,14 @@ int scratch_alloc(void** out, size_t bytes, cudaStream_t st)
     {
         std::lock_guard<std::mutex> lock(mu);
         if (!pools[dev]) {
+            // a pool cannot be created while the stream is being captured into a graph: this call then takes the
+            // device's default pool (make the first call of a process outside a capture to get the library's pool)
+            cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+            if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
+            if (cap != cudaStreamCaptureStatusNone) {
+                if (cudaMallocAsync(out, bytes, st) != cudaSuccess) { cudaGetLastError(); *out = nullptr; return INVCONV_CUDA_ERROR; }
+                return INVCONV_OK;
+            }
             cudaMemPoolProps props = {};
             props.allocType = cudaMemAllocationTypePinned;
             props.location.type = cudaMemLocationTypeDevice;
