@@ -48,7 +48,8 @@ enum invconv_status {
     INVCONV_UNSUPPORTED = 2,      /* k or C beyond the compiled limits, tensor too large */
     INVCONV_CUDA_ERROR = 3,       /* a launch or runtime call failed (cudaGetLastError) */
     INVCONV_TIMEOUT = 4,          /* a bounded device-side wait gave up (see invconv_get_status) */
-    INVCONV_WORKSPACE_TOO_SMALL = 5
+    INVCONV_WORKSPACE_TOO_SMALL = 5,
+    INVCONV_BOUNDS = 6            /* debug-bounds build only: a checked accessor caught an index outside its array */
 };
 
 /* Which kernel family serves a call.  AUTO picks by shape; the others force a
@@ -257,6 +258,16 @@ int invconv_probe_step_latency(int mechanism, int steps, unsigned long long* cyc
  * runs out, the kernel raises the device status word to INVCONV_TIMEOUT and returns normally; the context
  * stays usable.  invconv_get_status then reports INVCONV_TIMEOUT once. */
 int invconv_selftest_wait_timeout(unsigned limit_cycles, void* stream);
+
+/* Debug-bounds build (the tensor-core and flow-step kernels compiled with -DINVCONV_DEBUG_BOUNDS,
+ * libinvconv_b200_debug.so): every index those kernels compute for shared or global memory goes through a
+ * checked accessor; an index outside its array is recorded instead of used, and invconv_get_status reports
+ * INVCONV_BOUNDS.  invconv_debug_bounds_info fills info[0..3] = {site number, index, limit, number of
+ * violations} of the current device and clears the record; it returns INVCONV_UNSUPPORTED in the normal build.
+ * invconv_selftest_bounds hands the accessor an index outside its limit on purpose (no memory is touched), to
+ * show that the record and the status work; INVCONV_UNSUPPORTED in the normal build. */
+int invconv_debug_bounds_info(int* info /* host, 4 ints */);
+int invconv_selftest_bounds(void* stream);
 
 /* Development and test controls -- not needed in normal use.  They force one of two equivalent kernels or
  * launch modes so that tests and measurements can compare them; results are the same within rounding.

@@ -16,7 +16,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libinvconv_b200.so")
 
-OK, BAD_ARG, UNSUPPORTED, CUDA_ERROR, TIMEOUT, WORKSPACE_TOO_SMALL = range(6)
+OK, BAD_ARG, UNSUPPORTED, CUDA_ERROR, TIMEOUT, WORKSPACE_TOO_SMALL, BOUNDS = range(7)
 PATH_AUTO, PATH_GENERIC, PATH_WARP, PATH_TEAM, PATH_TENSOR = range(5)
 WS_CONTROL_BYTES = 256
 
@@ -63,6 +63,10 @@ def lib() -> ctypes.CDLL:
         L.invconv_set_option.argtypes = [ci, ci]
         L.invconv_set_option.restype = ci
         L.invconv_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp]
+        L.invconv_debug_bounds_info.argtypes = [ctypes.POINTER(ci)]
+        L.invconv_debug_bounds_info.restype = ci
+        L.invconv_selftest_bounds.argtypes = [vp]
+        L.invconv_selftest_bounds.restype = ci
         L.invconv_selftest_wait_timeout.restype = ci
         L.invconv_path_for.argtypes = [ci] * 5
         L.invconv_cluster_size_for.argtypes = [ci] * 5
@@ -323,6 +327,16 @@ def invconv_selftest_wait_timeout(limit_cycles: int = 20000, stream: Optional[to
     with torch.cuda.device(device):
         _check(lib().invconv_selftest_wait_timeout(limit_cycles, _stream_ptr(stream, device)),
                "invconv_selftest_wait_timeout")
+
+
+def invconv_debug_bounds_info():
+    """(site, index, limit, count) of the debug-bounds build's record (cleared by the call); None in the normal build."""
+    arr = (ctypes.c_int * 4)()
+    rc = int(lib().invconv_debug_bounds_info(arr))
+    if rc == UNSUPPORTED:
+        return None
+    _check(rc, "invconv_debug_bounds_info")
+    return tuple(int(v) for v in arr)
 
 
 def invconv_set_path(path: int) -> int:

@@ -76,5 +76,30 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+LIB_DEBUG = os.path.join(PKG, "libinvconv_b200_debug.so")
+
+
+def build_debug_bounds() -> str:
+    """The debug-bounds variant: the tensor-core and flow-step translation units recompiled with
+    -DINVCONV_DEBUG_BOUNDS (checked accessors) and linked with the regular objects of the rest."""
+    build()
+    objdir = os.path.join(PKG, "build")
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC",
+             "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-DINVCONV_DEBUG_BOUNDS"]
+    procs, objs = [], [os.path.join(objdir, "invconv_lib.o")]
+    for name in ("tensor_lib", "flow_step_lib"):
+        obj = os.path.join(objdir, name + "_dbg.o")
+        objs.append(obj)
+        procs.append(subprocess.Popen([NVCC, "-c", *flags, os.path.join(CSRC, name + ".cu"), "-o", obj]))
+    if any(pr.wait() != 0 for pr in procs):
+        raise RuntimeError("nvcc failed for the debug-bounds build")
+    tmp = LIB_DEBUG + f".tmp{os.getpid()}"
+    subprocess.check_call([NVCC, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-Xcompiler", "-fPIC", *objs, "-o", tmp])
+    os.replace(tmp, LIB_DEBUG)
+    return LIB_DEBUG
+
+
 if __name__ == "__main__":
     print(build(force=True, verbose="-v" in sys.argv))
+    if "--debug-bounds" in sys.argv:
+        print(build_debug_bounds())

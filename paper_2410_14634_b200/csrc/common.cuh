@@ -19,6 +19,26 @@ static __device__ int g_device_status = 0;
 
 __device__ __forceinline__ void raise_status(int code) { atomicMax(&g_device_status, code); }
 
+// Checked accessors (development build, -DINVCONV_DEBUG_BOUNDS; stands in for a memory checker): an index
+// that is about to be used goes through INVCONV_CHECKED(index, limit, site).  In the debug build an index outside
+// [0, limit) is recorded (the first one with its site number, index and limit; a count of all), the status word
+// is raised to INVCONV_BOUNDS and the macro yields false, so the caller skips the access instead of faulting.
+// In the normal build the macro is the constant true and costs nothing.
+#ifdef INVCONV_DEBUG_BOUNDS
+static __device__ int g_bounds_record[4] = {0, 0, 0, 0};      // site, index, limit, count
+__device__ __forceinline__ bool bounds_ok(long long i, long long n, int site)
+{
+    if (i >= 0 && i < n) return true;
+    atomicAdd(&g_bounds_record[3], 1);
+    if (atomicCAS(&g_bounds_record[0], 0, site) == 0) { g_bounds_record[1] = (int)i; g_bounds_record[2] = (int)n; }
+    raise_status(INVCONV_BOUNDS);
+    return false;
+}
+#define INVCONV_CHECKED(i, n, site) (::invconv::bounds_ok((long long)(i), (long long)(n), (site)))
+#else
+#define INVCONV_CHECKED(i, n, site) (true)
+#endif
+
 // Index helpers.  Activations are [B][C][H][W]; kernels [C][C][k][k].
 __host__ __device__ __forceinline__ size_t act_index(int n, int c, int h, int w, int C, int H, int W) {
     return (((size_t)n * C + c) * H + h) * W + w;

@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(kConvTensorThreads, 1) conv_tensor_kernel(cons
                 const int w = e % W, hr = (e / W) % rows, chunk = e / (W * rows);
                 const int h = h0 - (K - 1) + hr;
                 float v[8];
-                if (h >= 0 && h < H) {
+                if (h >= 0 && h < H && INVCONV_CHECKED((size_t)n * C * HW + (size_t)(chunk * 8 + 7) * HW + h * W + w, (size_t)p.B * C * HW, 302)) {
                     const float* src = xn + (size_t)(chunk * 8) * HW + h * W + w;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[j] = __ldg(src + (size_t)j * HW);
@@ -129,6 +129,7 @@ __global__ void __launch_bounds__(kConvTensorThreads, 1) conv_tensor_kernel(cons
                 for (int j = 0; j < 8; ++j) hi[j] = tf32_hi(v[j]);
                 unsigned char* cb = s_x + (size_t)chunk * chunk_bytes;
                 const int slot = FRONT + hr * Wp + w + K - 1;
+                if (!INVCONV_CHECKED(slot, SL, 301)) continue;
                 *reinterpret_cast<float4*>(cb + ((size_t)0 * SL + slot) * 16) = make_float4(hi[0], hi[1], hi[2], hi[3]);
                 *reinterpret_cast<float4*>(cb + ((size_t)1 * SL + slot) * 16) = make_float4(hi[4], hi[5], hi[6], hi[7]);
                 const __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
@@ -160,7 +161,7 @@ __global__ void __launch_bounds__(kConvTensorThreads, 1) conv_tensor_kernel(cons
                     umma::tmem_ld16(lane_addr + (uint32_t)(C + c0), a1);
                     umma::tmem_ld_fence(a0);
                     umma::tmem_ld_fence(a1);
-                    if (valid) {
+                    if (valid && INVCONV_CHECKED((dst - p.y) + (size_t)(c0 + 15) * HW, (size_t)p.B * C * HW, 303)) {
 #pragma unroll
                         for (int j = 0; j < 16; ++j) dst[(size_t)(c0 + j) * HW] = __uint_as_float(a0[j]) + __uint_as_float(a1[j]);
                     }
@@ -189,6 +190,7 @@ __global__ void __launch_bounds__(kConvTensorThreads, 1) conv_tensor_kernel(cons
                     umma::fence_after_sync();
                     const int dh = tap / K, dw = tap - dh * K;
                     const uint32_t row0 = (uint32_t)(FRONT + (K - 1 - dh) * Wp - dw) * 16;
+                    (void)INVCONV_CHECKED(FRONT + (K - 1 - dh) * Wp - dw + 127, SL, 304);
                     for (int ch = 0; ch < nchunk; ++ch) {
                         const uint32_t xb = xa + (uint32_t)ch * chunk_bytes + row0;
                         const uint32_t wb = wa + (uint32_t)stage * p.wstage_bytes + (uint32_t)ch * 4 * C * 16;

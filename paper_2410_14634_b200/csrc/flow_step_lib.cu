@@ -57,7 +57,8 @@ __global__ void __launch_bounds__(256) flow_mix_kernel(const float* __restrict__
         const int o = e / kMixPixels, p = e - o * kMixPixels;
         float acc = cb[o];
         for (int c = 0; c < C; ++c) acc = fmaf(A[o * (C + 1) + c], tile[c * kMixPixels + p], acc);
-        if (p < np) dst[(size_t)o * HW + p] = acc;
+        if (p < np && INVCONV_CHECKED((size_t)n * C * HW + t0 + (size_t)o * HW + p, (size_t)gridDim.x / tiles * C * HW, 401))
+            dst[(size_t)o * HW + p] = acc;
     }
 }
 
@@ -211,6 +212,34 @@ int launch_mix(const float* in, const float* V, const float* s, const float* b, 
 }
 
 }  // namespace
+
+namespace invconv_internal {
+
+int flow_read_clear_status(int* status_out)
+{
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return INVCONV_CUDA_ERROR; }
+    if (v != 0) {
+        const int zero = 0;
+        cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int));
+    }
+    *status_out = v;
+    return INVCONV_OK;
+}
+
+int flow_bounds_info(int* info)
+{
+#ifdef INVCONV_DEBUG_BOUNDS
+    const int zero[4] = {0, 0, 0, 0};
+    if (cudaMemcpyFromSymbol(info, g_bounds_record, 4 * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return INVCONV_CUDA_ERROR; }
+    cudaMemcpyToSymbol(g_bounds_record, zero, sizeof(zero));
+#else
+    info[0] = info[1] = info[2] = info[3] = 0;
+#endif
+    return INVCONV_OK;
+}
+
+}  // namespace invconv_internal
 
 extern "C" {
 

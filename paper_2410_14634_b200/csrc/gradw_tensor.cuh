@@ -115,7 +115,8 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
                 for (int j = 0; j < 4; ++j) {
                     a[j] = b1[j] = b0[j] = make_float4(0.f, 0.f, 0.f, 0.f);
                     const int h = r * RB + hl_[j0 + j];
-                    if (goff[j0 + j] >= 0 && h < H) {
+                    if (goff[j0 + j] >= 0 && h < H &&
+                        INVCONV_CHECKED((size_t)n * C * HW + (size_t)r * RB * W + goff[j0 + j] + 3, (size_t)p.B * C * HW, 202)) {
                         a[j] = __ldg(reinterpret_cast<const float4*>(gyb + goff[j0 + j]));
                         if (h >= dh) {
                             b1[j] = __ldg(reinterpret_cast<const float4*>(xb + goff[j0 + j]));
@@ -136,6 +137,7 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     if (goff[j0 + j] < 0) continue;
+                    if (!INVCONV_CHECKED(soff[j0 + j] + 15, copy_bytes, 201)) continue;
                     unsigned char* da_ = sa + soff[j0 + j];
                     unsigned char* db_ = sb + soff[j0 + j];
                     *reinterpret_cast<float4*>(da_) = make_float4(tf32_hi(a[j].x), tf32_hi(a[j].y), tf32_hi(a[j].z), tf32_hi(a[j].w));
@@ -164,7 +166,7 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
                     uint32_t v[16];
                     umma::tmem_ld16(lane_addr + (uint32_t)(dw * C + c0), v);
                     umma::tmem_ld_fence(v);
-                    if (co < C) {
+                    if (co < C && INVCONV_CHECKED((dst - p.partials) + c0 + 15, (size_t)p.S * K * K * C * C, 203)) {
 #pragma unroll
                         for (int j = 0; j < 16; j += 4)
                             *reinterpret_cast<float4*>(dst + c0 + j) =

@@ -1116,6 +1116,17 @@ int invconv_set_path(int path)
     return g_forced_path.exchange(path);
 }
 
+int invconv_debug_bounds_info(int* info)
+{
+    if (!info) return INVCONV_BAD_ARG;
+    return invconv_internal::tensor_bounds_info(info);
+}
+
+int invconv_selftest_bounds(void* stream)
+{
+    return invconv_internal::tensor_selftest_bounds(as_stream(stream));
+}
+
 int invconv_set_option(int option, int value)
 {
     if (option < 0 || option >= INVCONV_OPT_COUNT) return -1;
@@ -1156,6 +1167,9 @@ int invconv_get_status(void* stream, int* device_status_out)
         cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int));
     }
     if (invconv_internal::tensor_read_clear_status(&vt) != INVCONV_OK) return INVCONV_CUDA_ERROR;
+    int vf = 0;
+    if (invconv_internal::flow_read_clear_status(&vf) != INVCONV_OK) return INVCONV_CUDA_ERROR;
+    if (vf > vt) vt = vf;
     *device_status_out = v > vt ? v : vt;
     return INVCONV_OK;
 }
@@ -1191,6 +1205,7 @@ const char* invconv_status_string(int status)
     case INVCONV_CUDA_ERROR: return "CUDA error";
     case INVCONV_TIMEOUT: return "device-side wait timed out";
     case INVCONV_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case INVCONV_BOUNDS: return "checked accessor caught an index out of bounds (debug-bounds build)";
     default: return "unknown status";
     }
 }

@@ -43,6 +43,10 @@ int warp_step_backward(const float* grad_u, const float* x, const float* w, cons
 int tensor_launch(const invconv::TensorPlan& pl, bool bwd, const float* rhs, const float* w, float* out,
                   invconv::Geom g, float* A, unsigned char* wop, cudaStream_t st, float* logdet_out = nullptr);
 int tensor_read_clear_status(int* status_out);
+int flow_read_clear_status(int* status_out);              // flow_step_lib.cu's copy of the status word
+int tensor_bounds_info(int* info);                        // debug-bounds build: first violation and count (both units)
+int flow_bounds_info(int* info);
+int tensor_selftest_bounds(cudaStream_t st);
 
 // tensor_lib.cu: y = f(x) on the tensor cores; `pack` is device scratch of pl.pack_bytes bytes.
 int conv_tensor_launch(const invconv::ConvTensorPlan& pl, const float* x, const float* w, float* y, invconv::Geom g,

@@ -88,6 +88,7 @@ __device__ __forceinline__ void wait_bar(unsigned long long* bar, unsigned parit
 // `chunk_base` is the shared-memory address of the chunk's block [kind][plane][rows][16 B].
 __device__ __forceinline__ void store_operand_row(unsigned char* chunk_base, int rows, int row, const float (&v)[8])
 {
+    if (!INVCONV_CHECKED(row, rows, 101)) return;
     float hi[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) hi[j] = tf32_hi(v[j]);
@@ -206,6 +207,7 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
                 umma::fence_after_sync();
                 uint32_t acc[CG][8], own[4];
                 const uint32_t col = (uint32_t)(slot_d * C);
+                (void)INVCONV_CHECKED(col + C - 1, p.tmem_cols, 105);
                 slot_d = slot_d + 1 == S ? 0 : slot_d + 1;
 #pragma unroll
                 for (int q = 0; q < CG; ++q) umma::tmem_ld8(lane_addr + col + (wg * CG + q) * 8, acc[q]);
@@ -234,7 +236,8 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
                 float4 pa[R - 1];
 #pragma unroll
                 for (int sl = 0; sl < R - 1; ++sl)
-                    pa[sl] = on_diag ? *reinterpret_cast<const float4*>(recv_b + (size_t)sl * 128 * CS) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    pa[sl] = (on_diag && INVCONV_CHECKED((recv_b - s_recv) + (size_t)sl * 128 * CS + 3, 2 * recv_buf_floats, 102))
+                                 ? *reinterpret_cast<const float4*>(recv_b + (size_t)sl * 128 * CS) : make_float4(0.f, 0.f, 0.f, 0.f);
                 float v[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int pr = 0; pr < R; ++pr) {
@@ -256,6 +259,7 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
                 {   // this warpgroup's half of the operand row: tf32 plane wg, 8 bytes of each bf16 plane
                     unsigned char* xb = s_x + b * xbuf_bytes;
                     const int row = HALO + m;
+                    (void)INVCONV_CHECKED(row, ROWS, 101);
                     float hi[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) hi[j] = tf32_hi(v[j]);
@@ -270,8 +274,10 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
                 if (valid) {
                     const int hh = p.rot ? H - 1 - h : h, ww = p.rot ? W - 1 - w : w;
                     float* dst = s_stage + (size_t)i * p.stage_img + (size_t)(wg * 4) * H * W + (size_t)hh * W + ww;
+                    if (INVCONV_CHECKED((dst - s_stage) + (size_t)3 * H * W, (size_t)I * p.stage_img, 103)) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) dst[(size_t)j * H * W] = v[j];
+                        for (int j = 0; j < 4; ++j) dst[(size_t)j * H * W] = v[j];
+                    }
                 }
             }
             fence_proxy_async();          // the staged slice is stored by bulk copies
@@ -312,6 +318,8 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
                     if (c > MAXSLOTS) c = MAXSLOTS;
                     const uint32_t dcol = tmem + (uint32_t)(s0 * C);
                     const uint32_t nbits = ((uint32_t)(c * C) >> 3) << 17;
+                    if (!INVCONV_CHECKED((s0 + c) * C - 1, p.tmem_cols, 106) || !INVCONV_CHECKED(HALO - dh * I, ROWS - 127, 107) ||
+                        !INVCONV_CHECKED((a + c) * C - 1, KC, 108)) break;
                     umma::mma_tf32(dcol, atf, wd_tf + wrow + (uint32_t)(a * C), idesc_tf | nbits, 1u);
                     umma::mma_bf16(dcol, abf, wd_bf + wrow + (uint32_t)(a * C), idesc_bf | nbits, 1u);
                     a += c; n -= c; s0 += c;
@@ -373,8 +381,9 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
             if (lt == 0) {
                 mbar_expect_tx(ybar, (unsigned)nimg * slice_bytes);
                 for (int ii = 0; ii < nimg; ++ii)
-                    bulk_g2s(s_stage + (size_t)ii * p.stage_img,
-                             p.rhs + (size_t)(g * I + ii) * img_floats + (size_t)rank * CS * H * W, slice_bytes, ybar);
+                    if (INVCONV_CHECKED((size_t)(g * I + ii) * img_floats + (size_t)(rank + 1) * CS * H * W - 1, (size_t)p.B * img_floats, 109))
+                        bulk_g2s(s_stage + (size_t)ii * p.stage_img,
+                                 p.rhs + (size_t)(g * I + ii) * img_floats + (size_t)rank * CS * H * W, slice_bytes, ybar);
             }
             wait_bar(ybar, ng & 1, gave_up);
             const bool img_ok = i < nimg;
@@ -386,8 +395,9 @@ __global__ void __launch_bounds__(kTensorThreads, 1) tensor_wavefront_kernel(con
                 if (img_ok && h < H && w >= 0 && w < W) {
                     const int hh = p.rot ? H - 1 - h : h, ww = p.rot ? W - 1 - w : w;
                     const float* src = s_stage + (size_t)i * p.stage_img + (size_t)hh * W + ww;
+                    const bool inb = INVCONV_CHECKED((src - s_stage) + (size_t)(CS - 1) * H * W, (size_t)I * p.stage_img, 104);
 #pragma unroll
-                    for (int j = 0; j < CS; ++j) v[j] = src[(size_t)j * H * W];
+                    for (int j = 0; j < CS; ++j) v[j] = inb ? src[(size_t)j * H * W] : 0.f;
                 } else {
 #pragma unroll
                     for (int j = 0; j < CS; ++j) v[j] = 0.f;

@@ -138,6 +138,38 @@ int conv_tensor_launch(const ConvTensorPlan& pl, const float* x, const float* w,
     return check_launch();
 }
 
+#ifdef INVCONV_DEBUG_BOUNDS
+namespace { __global__ void bounds_selftest_kernel() { (void)INVCONV_CHECKED(5, 3, 999); } }
+#endif
+
+int tensor_selftest_bounds(cudaStream_t st)
+{
+#ifdef INVCONV_DEBUG_BOUNDS
+    bounds_selftest_kernel<<<1, 1, 0, st>>>();
+    return check_launch();
+#else
+    (void)st;
+    return INVCONV_UNSUPPORTED;
+#endif
+}
+
+int tensor_bounds_info(int* info)
+{
+#ifdef INVCONV_DEBUG_BOUNDS
+    int a[4] = {0, 0, 0, 0}, b[4] = {0, 0, 0, 0};
+    const int zero[4] = {0, 0, 0, 0};
+    if (cudaMemcpyFromSymbol(a, g_bounds_record, sizeof(a)) != cudaSuccess) { cudaGetLastError(); return INVCONV_CUDA_ERROR; }
+    cudaMemcpyToSymbol(g_bounds_record, zero, sizeof(zero));
+    if (flow_bounds_info(b) != INVCONV_OK) return INVCONV_CUDA_ERROR;
+    const int* first = a[0] ? a : b;
+    info[0] = first[0]; info[1] = first[1]; info[2] = first[2]; info[3] = a[3] + b[3];
+    return INVCONV_OK;
+#else
+    (void)info;
+    return INVCONV_UNSUPPORTED;
+#endif
+}
+
 int tensor_read_clear_status(int* status_out)
 {
     int v = 0;
