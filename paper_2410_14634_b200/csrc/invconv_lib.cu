@@ -723,8 +723,14 @@ int launch_forward(int path, const float* y, const float* w, float* x, Geom g,
         return launch_warp(false, y, w, x, nullptr, nullptr, g, ws, st, nullptr, logdet_out);
     case INVCONV_PATH_TEAM:
         return launch_team(false, y, w, x, g, ws, st, logdet_out);
-    case INVCONV_PATH_TENSOR:
+    case INVCONV_PATH_TENSOR: {
+        // buffers off a 16-byte boundary cannot use the bulk copies of the tensor family: the team family serves
+        // them from the same workspace (its layout is a prefix of the tensor family's)
+        const bool aligned = ((reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(x)) & 15) == 0;
+        if (!aligned && g_forced_path.load() == INVCONV_PATH_AUTO && team_plan(g.B, g.C, g.H, g.W, g.k).ok)
+            return launch_team(false, y, w, x, g, ws, st, logdet_out);
         return launch_tensor(false, y, w, x, g, ws, st, logdet_out);
+    }
     default:
         return INVCONV_UNSUPPORTED;
     }
@@ -765,7 +771,10 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
     }
     case INVCONV_PATH_TENSOR: {
         if (g.B > 0) {
-            const int rc = launch_tensor(true, gx, w, gy, g, ws, st);
+            const bool aligned = ((reinterpret_cast<uintptr_t>(gx) | reinterpret_cast<uintptr_t>(gy)) & 15) == 0;
+            const int rc = (!aligned && g_forced_path.load() == INVCONV_PATH_AUTO && team_plan(g.B, g.C, g.H, g.W, g.k).ok)
+                               ? launch_team(true, gx, w, gy, g, ws, st)
+                               : launch_tensor(true, gx, w, gy, g, ws, st);
             if (rc) return rc;
         }
         if (gw) return launch_gradw_tensor(gy, x, gw, g, ws, tensor_gradw_offset(g.B, g.C, g.H, g.W, g.k), st, ld);

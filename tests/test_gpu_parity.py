@@ -316,6 +316,35 @@ def test_a_bounded_wait_that_runs_out_is_reported_once_and_the_context_stays_usa
     assert nmax_err(x.cpu().numpy(), oracle.invconv_forward(y, w)) <= TOL_X
 
 
+@pytest.mark.parametrize("shape", [(3, 16, 8, 8, 3), (9, 48, 16, 16, 3)], ids=lambda s: "x".join(map(str, s)))
+def test_unaligned_buffers_on_shapes_of_the_tensor_family(B, oracle, shape):
+    """Buffers 4 bytes off a 16-byte boundary: the automatic choice must still serve the shape (the tensor family's
+    bulk copies need aligned slices, so another family takes over), forward, backward and masked convolution."""
+    import torch
+    Bn, C, H, W, k = shape
+    w, y, gx = workloads.make_custom(55 + sum(shape), Bn, C, H, W, k, sigma=0.05 / np.sqrt(C))
+
+    def off(a):
+        buf = torch.empty(a.size + 1, dtype=torch.float32, device="cuda")
+        v = buf[1:].view(a.shape)
+        v.copy_(torch.from_numpy(a))
+        return v
+
+    n = y.size
+    x = torch.empty(n + 1, dtype=torch.float32, device="cuda")[1:].view(y.shape)
+    gy = torch.empty(n + 1, dtype=torch.float32, device="cuda")[1:].view(y.shape)
+    yy = torch.empty(n + 1, dtype=torch.float32, device="cuda")[1:].view(y.shape)
+    B.invconv_forward(off(y), dev(w), out=x)
+    _, gw = B.invconv_backward(off(gx), x, dev(w), out_grad_y=gy)
+    B.masked_conv_forward(x, dev(w), out=yy)
+    torch.cuda.synchronize()
+    assert B.invconv_get_status() == 0
+    x_ref = oracle.invconv_forward(y, w)
+    gy_ref, gw_ref = oracle.invconv_backward(gx, x_ref, w)
+    assert nmax_err(x.cpu().numpy(), x_ref) <= TOL_X and nmax_err(gy.cpu().numpy(), gy_ref) <= TOL_X
+    assert nmax_err(gw.cpu().numpy(), gw_ref) <= TOL_GW and nmax_err(yy.cpu().numpy(), y) <= TOL_X
+
+
 def test_empty_batch_is_a_no_op_and_zeroes_grad_w(B):
     import torch
     w = dev(workloads.make_custom(9, 1, 2, 4, 4, 3)[0])
