@@ -149,6 +149,30 @@ int invconv_flow_step_backward(const float* grad_u, const float* x, const float*
                                const float* V, float* grad_y, float* grad_w, float* grad_s, float* grad_b, float* grad_V,
                                int B, int C, int H, int W, int k, void* stream);
 
+/* Reduced-precision storage variant of invconv_forward / invconv_backward: the activations y, x, grad_x and
+ * grad_y are bfloat16 in device memory ([B][C][H][W], contiguous, 2 bytes per value; passed as void*), the
+ * weights w and grad_w stay fp32.  Only the number format in memory changes: a bfloat16 value is widened
+ * exactly to fp32 when it is read, every sum of the method (the substitution chain of Section 3, Theorem 1's
+ * transposed solve, Theorem 2's correlation, which takes the fp32 grad_y before it is narrowed and the stored
+ * x) is carried in fp32 as in the fp32 calls, and an output is rounded to the nearest bfloat16 (ties to even)
+ * when it is written.  So x_stored = bf16(f^-1(y_stored)) up to the fp32 calls' own error, and the per-value
+ * error of an output is half a bfloat16 spacing (2^-9 relative) on top of that.  The paper has no such
+ * variant (it stores fp32); it halves the activation bytes per step for the batch-scaling regime of the
+ * paper's batch-size ablation.
+ *
+ * Shapes of the warp-shuffle family whose images fit shared memory read and write bfloat16 inside the
+ * wavefront kernel (C*H*W a multiple of 8, buffers 16-byte aligned, and -- backward with grad_w -- grad_w
+ * riding along in the wavefront): invconv_bf16_in_kernel says so for a shape.  Every other shape is composed:
+ * widen into fp32 scratch, the fp32 path, narrow the result -- same results, no bytes saved.
+ * Argument rules, errors and scratch (library-owned stream-ordered pool) as for invconv_forward / _backward. */
+int invconv_forward_bf16(const void* y_bf16, const float* w, void* x_bf16,
+                         int B, int C, int H, int W, int k, void* stream);
+int invconv_backward_bf16(const void* grad_x_bf16, const void* x_bf16, const float* w, void* grad_y_bf16, float* grad_w,
+                          int B, int C, int H, int W, int k, void* stream);
+/* 1 if the call above (backward != 0: invconv_backward_bf16, with_grad_w != 0: grad_w non-NULL) handles
+ * bfloat16 inside the wavefront kernel for this shape (given aligned buffers), 0 if it is composed. */
+int invconv_bf16_in_kernel(int B, int C, int H, int W, int k, int backward, int with_grad_w);
+
 /* Scratch bytes a forward or backward call of this shape needs (0 if none).
  * Same value for both directions. */
 size_t invconv_workspace_bytes(int B, int C, int H, int W, int k);

@@ -50,6 +50,12 @@ def lib() -> ctypes.CDLL:
         L.invconv_flow_step_forward.restype = ci
         L.invconv_flow_step_backward.argtypes = [fp] * 11 + [ci] * 5 + [vp]
         L.invconv_flow_step_backward.restype = ci
+        L.invconv_forward_bf16.argtypes = [vp, fp, vp, ci, ci, ci, ci, ci, vp]
+        L.invconv_forward_bf16.restype = ci
+        L.invconv_backward_bf16.argtypes = [vp, vp, fp, vp, fp, ci, ci, ci, ci, ci, vp]
+        L.invconv_backward_bf16.restype = ci
+        L.invconv_bf16_in_kernel.argtypes = [ci] * 7
+        L.invconv_bf16_in_kernel.restype = ci
         L.invconv_workspace_bytes.argtypes = [ci] * 5
         L.invconv_workspace_bytes.restype = sz
         L.invconv_forward_ws.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, vp, sz, vp]
@@ -274,6 +280,45 @@ def invconv_flow_step_backward(grad_u: torch.Tensor, x: torch.Tensor, w: torch.T
                                                 gV.data_ptr(), B, C, H, W, k, _stream_ptr(stream, x.device)),
                "invconv_flow_step_backward")
     return gy, gw, gs, gb, gV
+
+
+def _act16(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == 4 and t.is_contiguous()):
+        raise ValueError(f"{name} must be a contiguous bfloat16 CUDA tensor [B,C,H,W]")
+    return t
+
+
+def invconv_forward_bf16(y: torch.Tensor, w: torch.Tensor, out: Optional[torch.Tensor] = None,
+                         stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """x = f^{-1}(y) with bfloat16 activations in memory (fp32 weights, fp32 arithmetic)."""
+    _act16(y, "y")
+    B, C, H, W = y.shape
+    k = _kern(w, C)
+    x = torch.empty_like(y) if out is None else _act16(out, "out")
+    with torch.cuda.device(y.device):
+        _check(lib().invconv_forward_bf16(y.data_ptr(), w.data_ptr(), x.data_ptr(), B, C, H, W, k,
+                                          _stream_ptr(stream, y.device)), "invconv_forward_bf16")
+    return x
+
+
+def invconv_backward_bf16(grad_x: torch.Tensor, x: torch.Tensor, w: torch.Tensor, need_grad_w: bool = True,
+                          out_grad_y: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """(grad_y, grad_w) with bfloat16 activations in memory; grad_w is fp32 (None if not asked for)."""
+    _act16(grad_x, "grad_x")
+    _act16(x, "x")
+    B, C, H, W = x.shape
+    k = _kern(w, C)
+    gy = torch.empty_like(x) if out_grad_y is None else _act16(out_grad_y, "out_grad_y")
+    gw = torch.empty_like(w) if need_grad_w else None
+    with torch.cuda.device(x.device):
+        _check(lib().invconv_backward_bf16(grad_x.data_ptr(), x.data_ptr(), w.data_ptr(), gy.data_ptr(),
+                                           gw.data_ptr() if gw is not None else None, B, C, H, W, k,
+                                           _stream_ptr(stream, x.device)), "invconv_backward_bf16")
+    return gy, gw
+
+
+def invconv_bf16_in_kernel(B: int, C: int, H: int, W: int, k: int, backward: bool = False, with_grad_w: bool = True) -> bool:
+    return bool(lib().invconv_bf16_in_kernel(B, C, H, W, k, int(backward), int(with_grad_w)))
 
 
 class HostStep:

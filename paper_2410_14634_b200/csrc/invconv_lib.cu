@@ -3,6 +3,7 @@
 // below; nothing here computes.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstdlib>
@@ -249,15 +250,19 @@ struct WarpMix {
     bool grad_in = false;       // backward
 };
 
+// `bf16`: rhs, out and xsaved are bfloat16 images (see WarpParams::bf16); INVCONV_UNSUPPORTED where the kernel
+// cannot take them (images in global memory, grad_w from the separate kernel, sizes or pointers the bulk copies
+// do not accept) -- the caller then converts around the fp32 path.
 int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const float* xsaved, float* gw, Geom g,
                 void* ws, cudaStream_t st, const WarpMix* mix = nullptr, float* logdet_out = nullptr,
-                const LogdetFuse& ld = LogdetFuse{})
+                const LogdetFuse& ld = LogdetFuse{}, bool bf16 = false)
 {
     const WarpPlan pl = plan_warp(g.B, g.C, g.H, g.W, g.k, bwd);
     if (!pl.ok) return INVCONV_UNSUPPORTED;
     if (mix && pl.glb) return INVCONV_UNSUPPORTED;       // images in global memory: the caller composes the step
     const GradWSmallPlan gs = (bwd && gw) ? gradw_small_plan(g.B, g.C, g.H, g.W, g.k) : GradWSmallPlan{};
     const bool separate = bwd && gw && ws && gradw_separate(pl, gs, g.C, g.k);
+    if (bf16 && (pl.glb || separate || mix)) return INVCONV_UNSUPPORTED;
     WarpParams prm;
     prm.rhs = rhs; prm.w = w; prm.out = out; prm.xsaved = xsaved; prm.grad_w = separate ? nullptr : gw;
     prm.counter = static_cast<unsigned*>(ws);
@@ -274,6 +279,10 @@ int launch_warp(bool bwd, const float* rhs, const float* w, float* out, const fl
     const bool aligned = ((reinterpret_cast<uintptr_t>(rhs) | reinterpret_cast<uintptr_t>(out) |
                            reinterpret_cast<uintptr_t>(xsaved)) & 15) == 0;
     prm.bulk = (aligned && chw % 4 == 0) ? 1 : 0;
+    if (bf16) {
+        if (!aligned || chw % 8 != 0) return INVCONV_UNSUPPORTED;
+        prm.bulk = 1; prm.bf16 = 1;
+    }
     prm.glb = pl.glb ? 1 : 0;
     prm.vec = (aligned && g.W % 4 == 0) ? 1 : 0;
     int rc = INVCONV_UNSUPPORTED;
@@ -826,6 +835,73 @@ StepSide* step_side()
     return &s;
 }
 
+// ---------------------------------------------------------------- bfloat16 storage around the fp32 path
+// Where a kernel family cannot take bfloat16 images itself, the variant is composed: widen into fp32 scratch, run
+// the fp32 path, narrow the result.  Eight values per thread where the buffers allow 16-byte accesses.
+__global__ void widen_bf16_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out, size_t n, int vec)
+{
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    if (vec) {
+        for (size_t u = (size_t)blockIdx.x * blockDim.x + threadIdx.x; u < n / 8; u += stride) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(in) + u);
+            float4* d = reinterpret_cast<float4*>(out) + 2 * u;
+            d[0] = make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u),
+                               __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
+            d[1] = make_float4(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xffff0000u),
+                               __uint_as_float(v.w << 16), __uint_as_float(v.w & 0xffff0000u));
+        }
+    } else {
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) out[i] = __bfloat162float(in[i]);
+    }
+}
+
+__global__ void narrow_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, size_t n, int vec)
+{
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    if (vec) {
+        for (size_t u = (size_t)blockIdx.x * blockDim.x + threadIdx.x; u < n / 8; u += stride) {
+            const float4 a = reinterpret_cast<const float4*>(in)[2 * u], b = reinterpret_cast<const float4*>(in)[2 * u + 1];
+            reinterpret_cast<uint4*>(out)[u] =
+                make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+        }
+    } else {
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) out[i] = __float2bfloat16_rn(in[i]);
+    }
+}
+
+int launch_widen(const void* in, float* out, size_t n, cudaStream_t st)
+{
+    const int vec = ((reinterpret_cast<uintptr_t>(in) & 15) == 0 && n % 8 == 0) ? 1 : 0;
+    const size_t items = vec ? n / 8 : n;
+    const int blocks = (int)std::min<size_t>((items + 255) / 256, (size_t)sm_count() * 8);
+    widen_bf16_kernel<<<blocks > 0 ? blocks : 1, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(in), out, n, vec);
+    return check_launch();
+}
+
+int launch_narrow(const float* in, void* out, size_t n, cudaStream_t st)
+{
+    const int vec = ((reinterpret_cast<uintptr_t>(out) & 15) == 0 && n % 8 == 0) ? 1 : 0;
+    const size_t items = vec ? n / 8 : n;
+    const int blocks = (int)std::min<size_t>((items + 255) / 256, (size_t)sm_count() * 8);
+    narrow_bf16_kernel<<<blocks > 0 ? blocks : 1, 256, 0, st>>>(in, static_cast<__nv_bfloat16*>(out), n, vec);
+    return check_launch();
+}
+
+// Whether the wavefront kernel itself reads and writes the bfloat16 images (no conversion pass, no fp32 copy).
+bool bf16_in_kernel(int B, int C, int H, int W, int k, bool bwd, bool with_gw)
+{
+    if (resolve_path(B, C, H, W, k) != INVCONV_PATH_WARP) return false;
+    const WarpPlan pl = plan_warp(B, C, H, W, k, bwd);
+    if (!pl.ok || pl.glb || ((size_t)C * H * W) % 8 != 0) return false;
+    if (bwd && with_gw) {
+        const GradWSmallPlan gs = gradw_small_plan(B, C, H, W, k);
+        if (gradw_separate(pl, gs, C, k)) return false;
+    }
+    return true;
+}
+
+inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
 }  // namespace
 
 namespace invconv_internal {
@@ -917,6 +993,82 @@ int invconv_backward(const float* grad_x, const float* x, const float* w, float*
     const int ra = sc.acquire(need, as_stream(stream));
     if (ra) return ra;
     return invconv_backward_ws(grad_x, x, w, grad_y, grad_w, B, C, H, W, k, sc.p, need, stream);
+}
+
+int invconv_bf16_in_kernel(int B, int C, int H, int W, int k, int backward, int with_grad_w)
+{
+    if (check_shape(B, C, H, W, k) != INVCONV_OK || B == 0) return 0;
+    return bf16_in_kernel(B, C, H, W, k, backward != 0, with_grad_w != 0) ? 1 : 0;
+}
+
+int invconv_forward_bf16(const void* y, const float* w, void* x, int B, int C, int H, int W, int k, void* stream)
+{
+    const int rc = check_shape(B, C, H, W, k);
+    if (rc) return rc;
+    if (B == 0) return w ? INVCONV_OK : INVCONV_BAD_ARG;
+    if (!y || !w || !x || y == x) return INVCONV_BAD_ARG;
+    const cudaStream_t st = as_stream(stream);
+    const Geom g{B, C, H, W, k};
+    const int path = resolve_path(B, C, H, W, k);
+    const size_t need = up256(std::max<size_t>(workspace_bytes_for(path, B, C, H, W, k), INVCONV_WS_CONTROL_BYTES));
+    if (path == INVCONV_PATH_WARP) {
+        StreamScratch sc;
+        const int ra = sc.acquire(need, st);
+        if (ra) return ra;
+        const int rw = launch_warp(false, static_cast<const float*>(y), w, static_cast<float*>(x), nullptr, nullptr, g, sc.p, st,
+                                   nullptr, nullptr, LogdetFuse{}, true);
+        if (rw != INVCONV_UNSUPPORTED) return rw;
+    }
+    const size_t n = (size_t)B * C * H * W, act = up256(n * sizeof(float));
+    StreamScratch sc;
+    const int ra = sc.acquire(need + 2 * act, st);
+    if (ra) return ra;
+    float* y32 = reinterpret_cast<float*>(static_cast<char*>(sc.p) + need);
+    float* x32 = reinterpret_cast<float*>(static_cast<char*>(sc.p) + need + act);
+    int r = launch_widen(y, y32, n, st);
+    if (!r) r = launch_forward(path, y32, w, x32, g, sc.p, need, st);
+    if (!r) r = launch_narrow(x32, x, n, st);
+    return r;
+}
+
+int invconv_backward_bf16(const void* grad_x, const void* x, const float* w, void* grad_y, float* grad_w,
+                          int B, int C, int H, int W, int k, void* stream)
+{
+    const int rc = check_shape(B, C, H, W, k);
+    if (rc) return rc;
+    const cudaStream_t st = as_stream(stream);
+    if (B == 0) {
+        if (!w) return INVCONV_BAD_ARG;
+        if (grad_w && cudaMemsetAsync(grad_w, 0, sizeof(float) * C * C * k * k, st) != cudaSuccess) {
+            cudaGetLastError();
+            return INVCONV_CUDA_ERROR;
+        }
+        return INVCONV_OK;
+    }
+    if (!grad_x || !x || !w || !grad_y || grad_x == grad_y || x == grad_y) return INVCONV_BAD_ARG;
+    const Geom g{B, C, H, W, k};
+    const int path = resolve_path(B, C, H, W, k);
+    const size_t need = up256(std::max<size_t>(workspace_bytes_for(path, B, C, H, W, k), INVCONV_WS_CONTROL_BYTES));
+    if (path == INVCONV_PATH_WARP) {
+        StreamScratch sc;
+        const int ra = sc.acquire(need, st);
+        if (ra) return ra;
+        const int rw = launch_warp(true, static_cast<const float*>(grad_x), w, static_cast<float*>(grad_y),
+                                   static_cast<const float*>(x), grad_w, g, sc.p, st, nullptr, nullptr, LogdetFuse{}, true);
+        if (rw != INVCONV_UNSUPPORTED) return rw;
+    }
+    const size_t n = (size_t)B * C * H * W, act = up256(n * sizeof(float));
+    StreamScratch sc;
+    const int ra = sc.acquire(need + 3 * act, st);
+    if (ra) return ra;
+    float* gx32 = reinterpret_cast<float*>(static_cast<char*>(sc.p) + need);
+    float* x32 = reinterpret_cast<float*>(static_cast<char*>(sc.p) + need + act);
+    float* gy32 = reinterpret_cast<float*>(static_cast<char*>(sc.p) + need + 2 * act);
+    int r = launch_widen(grad_x, gx32, n, st);
+    if (!r && grad_w) r = launch_widen(x, x32, n, st);
+    if (!r) r = launch_backward(path, gx32, x32, w, gy32, grad_w, g, sc.p, need, st);
+    if (!r) r = launch_narrow(gy32, grad_y, n, st);
+    return r;
 }
 
 int masked_conv_forward(const float* x, const float* w, float* y, int B, int C, int H, int W, int k, void* stream)

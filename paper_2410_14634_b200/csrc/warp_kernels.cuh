@@ -39,6 +39,7 @@
 #pragma once
 
 #include <cstdio>
+#include <cuda_bf16.h>
 
 #include "common.cuh"
 #include "tma.cuh"
@@ -72,6 +73,10 @@ struct WarpParams {
     int mix_in = 0;                 // backward: rhs holds grad_u; grad_x = s * (V^T grad_u) is formed after the load
     float* logdet_out = nullptr;    // forward: CTA 0 also writes the layer's log-det (one float)
     LogdetFuse ld;                  // backward: the log-det's term on the diagonal of grad_w
+    // Reduced-precision storage: rhs, out and xsaved point to bfloat16 images (C*H*W a multiple of 8, bulk copies,
+    // images resident in shared memory, no flow-step neighbours).  They are widened to fp32 once they have
+    // arrived in shared memory and narrowed again on the way out; every sum in between is fp32 as without it.
+    int bf16 = 0;
 };
 
 template <int C> struct ColVec;
@@ -827,6 +832,48 @@ struct WarpSmem {
     }
 };
 
+// bfloat16 images that arrived in the upper half of their fp32 regions, widened in place by the whole CTA.
+// Unit u = 8 consecutive values: 16 bytes of bfloat16 at byte 2*CHW + 16u become 32 bytes of fp32 at byte 32u,
+// which overwrites the bfloat16 units 2u - CHW/8 and 2u - CHW/8 + 1.  Units are taken in ascending passes of
+// blockDim.x, every pass reading all of its units before the barrier and writing after it: what a pass
+// overwrites has either been widened by an earlier pass or is read by this one before the barrier.
+__device__ __forceinline__ void widen_bf16_in_place(float* regions, int region_floats, int nregions, int CHW)
+{
+    const int units = CHW >> 3;
+    for (int u0 = 0; u0 < units; u0 += (int)blockDim.x) {
+        const int u = u0 + (int)threadIdx.x;
+        for (int r0 = 0; r0 < nregions; r0 += 4) {
+            uint4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                v[q] = make_uint4(0u, 0u, 0u, 0u);
+                if (r0 + q < nregions && u < units)
+                    v[q] = *reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(regions + (size_t)(r0 + q) * region_floats) +
+                                                           2 * (size_t)CHW + 16 * (size_t)u);
+            }
+            __syncthreads();
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (r0 + q < nregions && u < units) {
+                    // a bfloat16 is the upper half of the fp32 with the same value
+                    float4* d = reinterpret_cast<float4*>(regions + (size_t)(r0 + q) * region_floats) + 2 * u;
+                    d[0] = make_float4(__uint_as_float(v[q].x << 16), __uint_as_float(v[q].x & 0xffff0000u),
+                                       __uint_as_float(v[q].y << 16), __uint_as_float(v[q].y & 0xffff0000u));
+                    d[1] = make_float4(__uint_as_float(v[q].z << 16), __uint_as_float(v[q].z & 0xffff0000u),
+                                       __uint_as_float(v[q].w << 16), __uint_as_float(v[q].w & 0xffff0000u));
+                }
+            }
+        }
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);     // .x = lo in the low half
+    return *reinterpret_cast<const unsigned*>(&t);
+}
+
 template <int C, int K, bool BWD, bool MULTI, bool GLB = false, bool RING = false, bool CS = false>
 __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
 {
@@ -867,13 +914,20 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     // kernel has completed, so only its launch latency overlaps
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // the image's bulk copy goes out first; the kernel transform below overlaps its latency
+    const bool narrow = !GLB && p.bf16 != 0;
     if (!GLB && leader && p.bulk) {
         mbar_init(&bars[li], 1);
         fence_mbar_init();
-        const unsigned bytes = (unsigned)CHW * 4u;
+        const unsigned bytes = (unsigned)CHW * (narrow ? 2u : 4u);
         mbar_expect_tx(&bars[li], want_gw ? 2 * bytes : bytes);
-        bulk_g2s(img, p.rhs + (size_t)n * CHW, bytes, &bars[li]);
-        if (want_gw) bulk_g2s(xs, p.xsaved + (size_t)n * CHW, bytes, &bars[li]);
+        if (narrow) {
+            // bfloat16 images land in the upper half of their regions (see widen_bf16_in_place)
+            bulk_g2s(img + (CHW >> 1), reinterpret_cast<const __nv_bfloat16*>(p.rhs) + (size_t)n * CHW, bytes, &bars[li]);
+            if (want_gw) bulk_g2s(xs + (CHW >> 1), reinterpret_cast<const __nv_bfloat16*>(p.xsaved) + (size_t)n * CHW, bytes, &bars[li]);
+        } else {
+            bulk_g2s(img, p.rhs + (size_t)n * CHW, bytes, &bars[li]);
+            if (want_gw) bulk_g2s(xs, p.xsaved + (size_t)n * CHW, bytes, &bars[li]);
+        }
     }
     if (!GLB && has_img && !p.bulk) {
         const float* src = p.rhs + (size_t)n * CHW;
@@ -895,6 +949,16 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     if (has_img) {
         if (!GLB && p.bulk) ok = mbar_wait_bounded(&bars[li], 0);
         ok = __all_sync(0xffffffffu, ok);
+    }
+    if constexpr (!GLB) {
+        if (narrow) {
+            // every image of the CTA has to be there before the CTA-wide widening passes; a wait that gave up
+            // fails the whole CTA (its images are left unsolved, the status says so)
+            for (int l2 = 0; l2 < p.ipc; ++l2)
+                if (l2 != li && blockIdx.x * p.ipc + l2 < p.B && !mbar_wait_bounded(&bars[l2], 0)) ok = false;
+            ok = __syncthreads_and(ok ? 1 : 0) != 0;
+            if (ok) widen_bf16_in_place(smem + lay.img_off, lay.imgf, (want_gw ? 2 : 1) * p.ipc, CHW);
+        }
     }
     if constexpr (BWD && !GLB) {
         if (p.mix_in) {
@@ -943,7 +1007,16 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
     }
     __syncthreads();
 
-    if (!GLB && has_img) {
+    if (narrow && has_img) {
+        // narrow on the way out: eight values per 16-byte store
+        uint4* d16 = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)n * CHW);
+        const float4* s4 = reinterpret_cast<const float4*>(img);
+        for (int u = j * 32 + lane; u < (CHW >> 3); u += p.nb * 32) {
+            const float4 a = s4[2 * u], b = s4[2 * u + 1];
+            d16[u] = make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+        }
+    }
+    if (!GLB && has_img && !narrow) {
         float* dst = p.out + (size_t)n * CHW;
         if (p.bulk && CHW * 4 <= 16384) {
             // small image: plain 16-byte stores retire without a completion wait at the end of the kernel
@@ -1047,7 +1120,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
             }
         }
     }
-    if (!GLB && p.bulk && leader && CHW * 4 > 16384) bulk_wait_read0();
+    if (!GLB && p.bulk && leader && CHW * 4 > 16384 && !narrow) bulk_wait_read0();
 }
 
 // Dynamic shared memory the kernel needs for a launch shape.
