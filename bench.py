@@ -155,14 +155,17 @@ class DeviceStep:
     """Rotating sets of device buffers for one workload (larger than twice the L2 in total unless `warm`),
     and the CUDA graphs that replay forward / backward / both over them."""
 
-    def __init__(self, shape, w, y, gx, device, warm=False):
+    def __init__(self, shape, w, y, gx, device, warm=False, storage="f32"):
         import torch
         from paper_2410_14634_b200 import binding
         self.torch, self.b, self.shape, self.device = torch, binding, shape, device
-        per_set = 4 * 4 * shape.elements
+        self.narrow = storage == "bf16"          # activations held as bfloat16 (the storage variant's calls)
+        per_set = 4 * (2 if self.narrow else 4) * shape.elements
         self.nsets = 1 if warm else max(3, -(-2 * L2_BYTES // per_set) + 1)
         yd = torch.from_numpy(y).to(device)
         gxd = torch.from_numpy(gx).to(device)
+        if self.narrow:
+            yd, gxd = yd.to(torch.bfloat16), gxd.to(torch.bfloat16)
         self.w = torch.from_numpy(w).to(device)
         self.y = [yd.clone() for _ in range(self.nsets)]
         self.gx = [gxd.clone() for _ in range(self.nsets)]
@@ -174,18 +177,25 @@ class DeviceStep:
         # make sure x holds valid data in every set (backward-only graphs read it)
         with torch.cuda.stream(self.stream):
             for i in range(self.nsets):
-                binding.invconv_forward(self.y[i], self.w, out=self.x[i])
-            binding.masked_conv_forward(self.x[0], self.w, out=self.gy[0])     # first call outside any graph capture
+                self.fwd(i)
+            if not self.narrow:
+                binding.masked_conv_forward(self.x[0], self.w, out=self.gy[0])     # first call outside any graph capture
         self.stream.synchronize()
 
     def fwd(self, i):
-        self.b.invconv_forward(self.y[i], self.w, out=self.x[i])
+        if self.narrow:
+            self.b.invconv_forward_bf16(self.y[i], self.w, out=self.x[i])
+        else:
+            self.b.invconv_forward(self.y[i], self.w, out=self.x[i])
 
     def conv(self, i):
         self.b.masked_conv_forward(self.x[i], self.w, out=self.gy[i])
 
     def bwd(self, i):
-        self.b.invconv_backward(self.gx[i], self.x[i], self.w, out_grad_y=self.gy[i], out_grad_w=self.gw)
+        if self.narrow:
+            _, gw = self.b.invconv_backward_bf16(self.gx[i], self.x[i], self.w, out_grad_y=self.gy[i], out_grad_w=self.gw)
+        else:
+            self.b.invconv_backward(self.gx[i], self.x[i], self.w, out_grad_y=self.gy[i], out_grad_w=self.gw)
 
     def graph(self, what: str, nsteps: int):
         """Capture `nsteps` steps (walking the buffer sets) into one CUDA graph."""
@@ -455,6 +465,17 @@ def per_config_rows(binding, workloads, device, pk, t_step, sm_mhz, steps, warmu
                "masked_conv_hbm_frac": round(8.0 * shape.elements / (tc * 1e-6) / 1e9 / pk["hbm_gbs"], 4)}
         if "t_tensor_us" in bd:
             row["t_tensor_us"] = round(bd["t_tensor_us"], 3)
+        dims = (shape.B, shape.C, shape.H, shape.W, shape.k)
+        if binding.invconv_bf16_in_kernel(*dims, backward=False):
+            # the storage variant where the wavefront kernel itself reads and writes bfloat16 (half the activation bytes)
+            d16 = DeviceStep(shape, w, y, gx, device, storage="bf16")
+            ms_f16, _ = d16.time_graphs("fwd", steps, warmup)
+            ms_b16, _ = d16.time_graphs("bwd", steps, warmup)
+            del d16
+            torch.cuda.empty_cache()
+            row["bf16_storage"] = {"t_fwd_us": round(ms_f16 / steps * 1e3, 2), "t_bwd_us": round(ms_b16 / steps * 1e3, 2),
+                                   "t_hbm_us": round(bd["t_hbm_us"] / 2, 3),
+                                   "backward_in_kernel": bool(binding.invconv_bf16_in_kernel(*dims, backward=True))}
         rows.append(row)
     return rows
 

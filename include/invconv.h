@@ -169,6 +169,16 @@ int invconv_forward_bf16(const void* y_bf16, const float* w, void* x_bf16,
                          int B, int C, int H, int W, int k, void* stream);
 int invconv_backward_bf16(const void* grad_x_bf16, const void* x_bf16, const float* w, void* grad_y_bf16, float* grad_w,
                           int B, int C, int H, int W, int k, void* stream);
+/* The same two calls with caller-owned device scratch of at least invconv_bf16_workspace_bytes(...) bytes,
+ * 256-byte aligned, under the rules of invconv_forward_ws (control words zeroed once, left zero by every
+ * call, one call at a time per workspace); these forms allocate nothing.  For a shape handled inside the
+ * wavefront kernel the size covers that route only: with buffers off a 16-byte boundary such a call returns
+ * INVCONV_WORKSPACE_TOO_SMALL (use the forms above, or pass need + 3 fp32 copies of the activations). */
+size_t invconv_bf16_workspace_bytes(int B, int C, int H, int W, int k);
+int invconv_forward_bf16_ws(const void* y_bf16, const float* w, void* x_bf16, int B, int C, int H, int W, int k,
+                            void* workspace, size_t workspace_bytes, void* stream);
+int invconv_backward_bf16_ws(const void* grad_x_bf16, const void* x_bf16, const float* w, void* grad_y_bf16, float* grad_w,
+                             int B, int C, int H, int W, int k, void* workspace, size_t workspace_bytes, void* stream);
 /* 1 if the call above (backward != 0: invconv_backward_bf16, with_grad_w != 0: grad_w non-NULL) handles
  * bfloat16 inside the wavefront kernel for this shape (given aligned buffers), 0 if it is composed. */
 int invconv_bf16_in_kernel(int B, int C, int H, int W, int k, int backward, int with_grad_w);

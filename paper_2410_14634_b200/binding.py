@@ -56,6 +56,12 @@ def lib() -> ctypes.CDLL:
         L.invconv_backward_bf16.restype = ci
         L.invconv_bf16_in_kernel.argtypes = [ci] * 7
         L.invconv_bf16_in_kernel.restype = ci
+        L.invconv_bf16_workspace_bytes.argtypes = [ci] * 5
+        L.invconv_bf16_workspace_bytes.restype = sz
+        L.invconv_forward_bf16_ws.argtypes = [vp, fp, vp, ci, ci, ci, ci, ci, vp, sz, vp]
+        L.invconv_forward_bf16_ws.restype = ci
+        L.invconv_backward_bf16_ws.argtypes = [vp, vp, fp, vp, fp, ci, ci, ci, ci, ci, vp, sz, vp]
+        L.invconv_backward_bf16_ws.restype = ci
         L.invconv_workspace_bytes.argtypes = [ci] * 5
         L.invconv_workspace_bytes.restype = sz
         L.invconv_forward_ws.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, vp, sz, vp]
@@ -120,9 +126,11 @@ def _kern(w: torch.Tensor, C: int) -> int:
 _workspaces: dict = {}
 
 
-def workspace(B: int, C: int, H: int, W: int, k: int, device, stream_ptr: int) -> Optional[torch.Tensor]:
-    """A zero-initialised scratch tensor for this shape, cached per (device, stream)."""
-    need = int(lib().invconv_workspace_bytes(B, C, H, W, k))
+def workspace(B: int, C: int, H: int, W: int, k: int, device, stream_ptr: int, bf16: bool = False) -> Optional[torch.Tensor]:
+    """A zero-initialised scratch tensor for this shape, cached per (device, stream); `bf16`: sized for the
+    bfloat16-storage calls."""
+    size_of = lib().invconv_bf16_workspace_bytes if bf16 else lib().invconv_workspace_bytes
+    need = int(size_of(B, C, H, W, k))
     if need == 0:
         return None
     key = (torch.device(device).index, stream_ptr)
@@ -296,24 +304,37 @@ def invconv_forward_bf16(y: torch.Tensor, w: torch.Tensor, out: Optional[torch.T
     k = _kern(w, C)
     x = torch.empty_like(y) if out is None else _act16(out, "out")
     with torch.cuda.device(y.device):
-        _check(lib().invconv_forward_bf16(y.data_ptr(), w.data_ptr(), x.data_ptr(), B, C, H, W, k,
-                                          _stream_ptr(stream, y.device)), "invconv_forward_bf16")
+        sp = _stream_ptr(stream, y.device)
+        if (y.data_ptr() | x.data_ptr()) & 15 or B == 0:
+            # buffers off a 16-byte boundary: the library sizes its own scratch for the route it has to take
+            _check(lib().invconv_forward_bf16(y.data_ptr(), w.data_ptr(), x.data_ptr(), B, C, H, W, k, sp), "invconv_forward_bf16")
+        else:
+            ws = workspace(B, C, H, W, k, y.device, sp, bf16=True)
+            _check(lib().invconv_forward_bf16_ws(y.data_ptr(), w.data_ptr(), x.data_ptr(), B, C, H, W, k,
+                                                 ws.data_ptr(), ws.numel(), sp), "invconv_forward_bf16")
     return x
 
 
 def invconv_backward_bf16(grad_x: torch.Tensor, x: torch.Tensor, w: torch.Tensor, need_grad_w: bool = True,
-                          out_grad_y: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+                          out_grad_y: Optional[torch.Tensor] = None, out_grad_w: Optional[torch.Tensor] = None,
+                          stream: Optional[torch.cuda.Stream] = None):
     """(grad_y, grad_w) with bfloat16 activations in memory; grad_w is fp32 (None if not asked for)."""
     _act16(grad_x, "grad_x")
     _act16(x, "x")
     B, C, H, W = x.shape
     k = _kern(w, C)
     gy = torch.empty_like(x) if out_grad_y is None else _act16(out_grad_y, "out_grad_y")
-    gw = torch.empty_like(w) if need_grad_w else None
+    gw = (out_grad_w if out_grad_w is not None else torch.empty_like(w)) if need_grad_w else None
     with torch.cuda.device(x.device):
-        _check(lib().invconv_backward_bf16(grad_x.data_ptr(), x.data_ptr(), w.data_ptr(), gy.data_ptr(),
-                                           gw.data_ptr() if gw is not None else None, B, C, H, W, k,
-                                           _stream_ptr(stream, x.device)), "invconv_backward_bf16")
+        sp = _stream_ptr(stream, x.device)
+        gwp = gw.data_ptr() if gw is not None else None
+        if (grad_x.data_ptr() | x.data_ptr() | gy.data_ptr()) & 15 or B == 0:
+            _check(lib().invconv_backward_bf16(grad_x.data_ptr(), x.data_ptr(), w.data_ptr(), gy.data_ptr(), gwp,
+                                               B, C, H, W, k, sp), "invconv_backward_bf16")
+        else:
+            ws = workspace(B, C, H, W, k, x.device, sp, bf16=True)
+            _check(lib().invconv_backward_bf16_ws(grad_x.data_ptr(), x.data_ptr(), w.data_ptr(), gy.data_ptr(), gwp,
+                                                  B, C, H, W, k, ws.data_ptr(), ws.numel(), sp), "invconv_backward_bf16")
     return gy, gw
 
 

@@ -902,6 +902,12 @@ bool bf16_in_kernel(int B, int C, int H, int W, int k, bool bwd, bool with_gw)
 
 inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
+// The path's own workspace inside the storage variant's workspace (what follows it are the fp32 copies of a composed call).
+size_t bf16_ws_need(int path, int B, int C, int H, int W, int k)
+{
+    return up256(std::max<size_t>(workspace_bytes_for(path, B, C, H, W, k), INVCONV_WS_CONTROL_BYTES));
+}
+
 }  // namespace
 
 namespace invconv_internal {
@@ -1001,7 +1007,16 @@ int invconv_bf16_in_kernel(int B, int C, int H, int W, int k, int backward, int 
     return bf16_in_kernel(B, C, H, W, k, backward != 0, with_grad_w != 0) ? 1 : 0;
 }
 
-int invconv_forward_bf16(const void* y, const float* w, void* x, int B, int C, int H, int W, int k, void* stream)
+size_t invconv_bf16_workspace_bytes(int B, int C, int H, int W, int k)
+{
+    if (check_shape(B, C, H, W, k) != INVCONV_OK || B == 0) return 0;
+    const size_t need = bf16_ws_need(resolve_path(B, C, H, W, k), B, C, H, W, k);
+    const bool in_kernel = bf16_in_kernel(B, C, H, W, k, false, false) && bf16_in_kernel(B, C, H, W, k, true, true);
+    return need + (in_kernel ? 0 : 3 * up256((size_t)B * C * H * W * sizeof(float)));
+}
+
+int invconv_forward_bf16_ws(const void* y, const float* w, void* x, int B, int C, int H, int W, int k,
+                            void* workspace, size_t workspace_bytes, void* stream)
 {
     const int rc = check_shape(B, C, H, W, k);
     if (rc) return rc;
@@ -1010,29 +1025,25 @@ int invconv_forward_bf16(const void* y, const float* w, void* x, int B, int C, i
     const cudaStream_t st = as_stream(stream);
     const Geom g{B, C, H, W, k};
     const int path = resolve_path(B, C, H, W, k);
-    const size_t need = up256(std::max<size_t>(workspace_bytes_for(path, B, C, H, W, k), INVCONV_WS_CONTROL_BYTES));
+    const size_t need = bf16_ws_need(path, B, C, H, W, k);
+    if (!workspace || workspace_bytes < need) return INVCONV_WORKSPACE_TOO_SMALL;
     if (path == INVCONV_PATH_WARP) {
-        StreamScratch sc;
-        const int ra = sc.acquire(need, st);
-        if (ra) return ra;
-        const int rw = launch_warp(false, static_cast<const float*>(y), w, static_cast<float*>(x), nullptr, nullptr, g, sc.p, st,
+        const int rw = launch_warp(false, static_cast<const float*>(y), w, static_cast<float*>(x), nullptr, nullptr, g, workspace, st,
                                    nullptr, nullptr, LogdetFuse{}, true);
         if (rw != INVCONV_UNSUPPORTED) return rw;
     }
     const size_t n = (size_t)B * C * H * W, act = up256(n * sizeof(float));
-    StreamScratch sc;
-    const int ra = sc.acquire(need + 2 * act, st);
-    if (ra) return ra;
-    float* y32 = reinterpret_cast<float*>(static_cast<char*>(sc.p) + need);
-    float* x32 = reinterpret_cast<float*>(static_cast<char*>(sc.p) + need + act);
+    if (workspace_bytes < need + 2 * act) return INVCONV_WORKSPACE_TOO_SMALL;
+    float* y32 = reinterpret_cast<float*>(static_cast<char*>(workspace) + need);
+    float* x32 = reinterpret_cast<float*>(static_cast<char*>(workspace) + need + act);
     int r = launch_widen(y, y32, n, st);
-    if (!r) r = launch_forward(path, y32, w, x32, g, sc.p, need, st);
+    if (!r) r = launch_forward(path, y32, w, x32, g, workspace, need, st);
     if (!r) r = launch_narrow(x32, x, n, st);
     return r;
 }
 
-int invconv_backward_bf16(const void* grad_x, const void* x, const float* w, void* grad_y, float* grad_w,
-                          int B, int C, int H, int W, int k, void* stream)
+int invconv_backward_bf16_ws(const void* grad_x, const void* x, const float* w, void* grad_y, float* grad_w,
+                             int B, int C, int H, int W, int k, void* workspace, size_t workspace_bytes, void* stream)
 {
     const int rc = check_shape(B, C, H, W, k);
     if (rc) return rc;
@@ -1048,27 +1059,54 @@ int invconv_backward_bf16(const void* grad_x, const void* x, const float* w, voi
     if (!grad_x || !x || !w || !grad_y || grad_x == grad_y || x == grad_y) return INVCONV_BAD_ARG;
     const Geom g{B, C, H, W, k};
     const int path = resolve_path(B, C, H, W, k);
-    const size_t need = up256(std::max<size_t>(workspace_bytes_for(path, B, C, H, W, k), INVCONV_WS_CONTROL_BYTES));
+    const size_t need = bf16_ws_need(path, B, C, H, W, k);
+    if (!workspace || workspace_bytes < need) return INVCONV_WORKSPACE_TOO_SMALL;
     if (path == INVCONV_PATH_WARP) {
-        StreamScratch sc;
-        const int ra = sc.acquire(need, st);
-        if (ra) return ra;
         const int rw = launch_warp(true, static_cast<const float*>(grad_x), w, static_cast<float*>(grad_y),
-                                   static_cast<const float*>(x), grad_w, g, sc.p, st, nullptr, nullptr, LogdetFuse{}, true);
+                                   static_cast<const float*>(x), grad_w, g, workspace, st, nullptr, nullptr, LogdetFuse{}, true);
         if (rw != INVCONV_UNSUPPORTED) return rw;
     }
     const size_t n = (size_t)B * C * H * W, act = up256(n * sizeof(float));
-    StreamScratch sc;
-    const int ra = sc.acquire(need + 3 * act, st);
-    if (ra) return ra;
-    float* gx32 = reinterpret_cast<float*>(static_cast<char*>(sc.p) + need);
-    float* x32 = reinterpret_cast<float*>(static_cast<char*>(sc.p) + need + act);
-    float* gy32 = reinterpret_cast<float*>(static_cast<char*>(sc.p) + need + 2 * act);
+    if (workspace_bytes < need + 3 * act) return INVCONV_WORKSPACE_TOO_SMALL;
+    float* gx32 = reinterpret_cast<float*>(static_cast<char*>(workspace) + need);
+    float* x32 = reinterpret_cast<float*>(static_cast<char*>(workspace) + need + act);
+    float* gy32 = reinterpret_cast<float*>(static_cast<char*>(workspace) + need + 2 * act);
     int r = launch_widen(grad_x, gx32, n, st);
     if (!r && grad_w) r = launch_widen(x, x32, n, st);
-    if (!r) r = launch_backward(path, gx32, x32, w, gy32, grad_w, g, sc.p, need, st);
+    if (!r) r = launch_backward(path, gx32, x32, w, gy32, grad_w, g, workspace, need, st);
     if (!r) r = launch_narrow(gy32, grad_y, n, st);
     return r;
+}
+
+int invconv_forward_bf16(const void* y, const float* w, void* x, int B, int C, int H, int W, int k, void* stream)
+{
+    const int rc = check_shape(B, C, H, W, k);
+    if (rc) return rc;
+    if (B == 0) return w ? INVCONV_OK : INVCONV_BAD_ARG;
+    if (!y || !w || !x || y == x) return INVCONV_BAD_ARG;
+    const bool aligned = ((reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(x)) & 15) == 0;
+    const size_t bytes = bf16_ws_need(resolve_path(B, C, H, W, k), B, C, H, W, k) +
+                         ((aligned && bf16_in_kernel(B, C, H, W, k, false, false)) ? 0 : 2 * up256((size_t)B * C * H * W * sizeof(float)));
+    StreamScratch sc;
+    const int ra = sc.acquire(bytes, as_stream(stream));
+    if (ra) return ra;
+    return invconv_forward_bf16_ws(y, w, x, B, C, H, W, k, sc.p, bytes, stream);
+}
+
+int invconv_backward_bf16(const void* grad_x, const void* x, const float* w, void* grad_y, float* grad_w,
+                          int B, int C, int H, int W, int k, void* stream)
+{
+    const int rc = check_shape(B, C, H, W, k);
+    if (rc) return rc;
+    if (B == 0 || !grad_x || !x || !w || !grad_y || grad_x == grad_y || x == grad_y)
+        return invconv_backward_bf16_ws(grad_x, x, w, grad_y, grad_w, B, C, H, W, k, nullptr, 0, stream);
+    const bool aligned = ((reinterpret_cast<uintptr_t>(grad_x) | reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(grad_y)) & 15) == 0;
+    const size_t bytes = bf16_ws_need(resolve_path(B, C, H, W, k), B, C, H, W, k) +
+                         ((aligned && bf16_in_kernel(B, C, H, W, k, true, grad_w != nullptr)) ? 0 : 3 * up256((size_t)B * C * H * W * sizeof(float)));
+    StreamScratch sc;
+    const int ra = sc.acquire(bytes, as_stream(stream));
+    if (ra) return ra;
+    return invconv_backward_bf16_ws(grad_x, x, w, grad_y, grad_w, B, C, H, W, k, sc.p, bytes, stream);
 }
 
 int masked_conv_forward(const float* x, const float* w, float* y, int B, int C, int H, int W, int k, void* stream)

@@ -868,6 +868,42 @@ __device__ __forceinline__ void widen_bf16_in_place(float* regions, int region_f
     __syncthreads();
 }
 
+// The same for one image (and, with `second`, the saved image beside it) by the one warp that owns it: passes of
+// 128 units, four per lane, with a warp barrier between a pass's reads and its writes.
+__device__ __forceinline__ void widen_bf16_warp(float* region, float* second, int CHW, int lane)
+{
+    const int units = CHW >> 3;
+    for (int u0 = 0; u0 < units; u0 += 128) {
+        uint4 v[2][4];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const unsigned char* src = reinterpret_cast<const unsigned char*>(r == 0 ? region : second) + 2 * (size_t)CHW;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int u = u0 + q * 32 + lane;
+                v[r][q] = make_uint4(0u, 0u, 0u, 0u);
+                if ((r == 0 || second != nullptr) && u < units) v[r][q] = *reinterpret_cast<const uint4*>(src + 16 * (size_t)u);
+            }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            float4* dst = reinterpret_cast<float4*>(r == 0 ? region : second);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int u = u0 + q * 32 + lane;
+                if ((r == 0 || second != nullptr) && u < units) {
+                    dst[2 * u] = make_float4(__uint_as_float(v[r][q].x << 16), __uint_as_float(v[r][q].x & 0xffff0000u),
+                                             __uint_as_float(v[r][q].y << 16), __uint_as_float(v[r][q].y & 0xffff0000u));
+                    dst[2 * u + 1] = make_float4(__uint_as_float(v[r][q].z << 16), __uint_as_float(v[r][q].z & 0xffff0000u),
+                                                 __uint_as_float(v[r][q].w << 16), __uint_as_float(v[r][q].w & 0xffff0000u));
+                }
+            }
+        }
+        __syncwarp();
+    }
+}
+
 __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
 {
     const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);     // .x = lo in the low half
@@ -951,7 +987,10 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
         ok = __all_sync(0xffffffffu, ok);
     }
     if constexpr (!GLB) {
-        if (narrow) {
+        if (narrow && p.nb == 1) {
+            // one warp per image: it widens its own image as soon as that has arrived
+            if (has_img && ok) widen_bf16_warp(img, want_gw ? xs : nullptr, CHW, lane);
+        } else if (narrow) {
             // every image of the CTA has to be there before the CTA-wide widening passes; a wait that gave up
             // fails the whole CTA (its images are left unsolved, the status says so)
             for (int l2 = 0; l2 < p.ipc; ++l2)

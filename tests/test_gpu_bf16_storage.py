@@ -98,6 +98,54 @@ def test_bf16_storage_agrees_with_the_fp32_calls_on_the_same_values():
         assert torch.equal(gw16, gw32)
 
 
+def test_bf16_storage_with_buffers_off_a_16_byte_boundary():
+    """Buffers 2 bytes off: the wavefront kernel's bulk copies cannot take them, the composed route serves them."""
+    import torch
+    from paper_2410_14634_b200 import binding
+    from oracle import api as oracle
+    for shape in [(6, 3, 32, 32, 3), (9, 48, 16, 16, 3)]:
+        Bn, C, H, W, k = shape
+        w, y, gx = workloads.make_custom(31 + sum(shape), Bn, C, H, W, k, sigma=0.05 / np.sqrt(C))
+        wd = torch.from_numpy(w).cuda()
+
+        def off(a=None):
+            buf = torch.empty(y.size + 1, dtype=torch.bfloat16, device="cuda")
+            v = buf[1:].view(y.shape)
+            if a is not None:
+                v.copy_(torch.from_numpy(a))
+            return v
+
+        y16, gx16, x16, gy16 = off(y), off(gx), off(), off()
+        binding.invconv_forward_bf16(y16, wd, out=x16)
+        _, gw = binding.invconv_backward_bf16(gx16, x16, wd, out_grad_y=gy16)
+        torch.cuda.synchronize()
+        assert binding.invconv_get_status() == 0
+        check_stored(as64(x16), oracle.invconv_forward(as64(y16), w), "x")
+        gy_ref, gw_ref = oracle.invconv_backward(as64(gx16), as64(x16), w)
+        check_stored(as64(gy16), gy_ref, "grad_y")
+        assert nmax_err(gw.cpu().numpy(), gw_ref) <= 1e-3
+
+
+def test_bf16_workspace_forms_reject_a_short_workspace():
+    import torch
+    from paper_2410_14634_b200 import binding
+    L = binding.lib()
+    for shape in [(6, 3, 32, 32, 3), (4, 12, 16, 16, 3)]:
+        Bn, C, H, W, k = shape
+        need = L.invconv_bf16_workspace_bytes(*shape)
+        assert need >= L.invconv_workspace_bytes(*shape) > 0
+        ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+        y = torch.zeros(Bn, C, H, W, device="cuda", dtype=torch.bfloat16)
+        x = torch.empty_like(y)
+        w = torch.eye(C, device="cuda").reshape(C, C, 1, 1).repeat(1, 1, k, k).contiguous()
+        assert L.invconv_forward_bf16_ws(y.data_ptr(), w.data_ptr(), x.data_ptr(), *shape, ws.data_ptr(), need, None) == binding.OK
+        assert L.invconv_forward_bf16_ws(y.data_ptr(), w.data_ptr(), x.data_ptr(), *shape, ws.data_ptr(), 128, None) == binding.WORKSPACE_TOO_SMALL
+        assert L.invconv_backward_bf16_ws(y.data_ptr(), x.data_ptr(), w.data_ptr(), y.data_ptr(), None, *shape, ws.data_ptr(), need, None) == binding.BAD_ARG
+        gy = torch.empty_like(y)
+        assert L.invconv_backward_bf16_ws(y.data_ptr(), x.data_ptr(), w.data_ptr(), gy.data_ptr(), None, *shape, None, 0, None) == binding.WORKSPACE_TOO_SMALL
+        torch.cuda.synchronize()
+
+
 def test_bf16_storage_empty_batch_and_bad_arguments():
     import torch
     from paper_2410_14634_b200 import binding
