@@ -589,11 +589,10 @@ int launch_team(bool bwd, const float* rhs, const float* w, float* out, Geom g, 
     if (!pl.ok) return INVCONV_UNSUPPORTED;
     float* A = reinterpret_cast<float*>(static_cast<char*>(ws) + INVCONV_WS_CONTROL_BYTES);
     {
-        const size_t sm = team_solve_smem(g.C, g.k);
-        auto kern = bwd ? team_solve_kernel<true> : team_solve_kernel<false>;
-        const int rc = set_smem_limit(kern, sm);
-        if (rc) return rc;
-        kern<<<g.C + (g.C + 31) / 32, 512, sm, st>>>(w, A, g.C, g.k, nullptr, 0, 0u, logdet_out, g.H * g.W);
+        if (team_solve_launch(bwd, w, A, g.C, g.k, nullptr, 0, 0u, logdet_out, g.H * g.W, st) != cudaSuccess) {
+            cudaGetLastError();
+            return INVCONV_CUDA_ERROR;
+        }
         const int rl = check_launch();
         if (rl) return rl;
     }

@@ -40,17 +40,27 @@ namespace cg = cooperative_groups;
 //   forward : tap 0 -> L^-1[a][b];   tap != 0 -> sum_m L^-1[a][m] w[m][b][K-1-dh][K-1-dw]
 //   backward: tap 0 -> L^-1[b][a];   tap != 0 -> sum_m L^-1[m][a] w[b][m][K-1-dh][K-1-dw]
 // L = w[:, :, K-1, K-1] restricted to ci <= co.
-// One CTA per input channel b (plus CTAs for tap 0) solves  T S = RHS  by blocked right-looking substitution
-// in shared memory, T = L (forward, rows ascending) or L^T (backward, rows descending):
+// One CTA per input channel b (plus CTAs for tap 0) solves  T S = RHS  by substitution,
+// T = L (forward, rows ascending) or L^T (backward, rows descending):
 //   b <  C : RHS[m][kk] = w[m][b][kk] (forward) / w[b][m][kk] (backward); S[a][kk] -> A[flip(kk)][b][a]
 //   b >= C : RHS = 32 columns of the identity;                            S[a][b'] -> A[0][b'][a]
-// Pivot blocks of eight rows: every thread (row lane, column) first solves the block's 8x8 triangle for its
-// column in registers (redundantly across row lanes: 28 FMAs), then subtracts the block's contribution from
-// its share of the rows behind the block -- one block barrier per eight rows instead of one per row (the
-// barrier and its shared-memory round trip were the cost: 0.4 us per row at C = 48).  Solved rows go to a
-// separate array so that no thread reads a row another thread is rewriting.
+// The columns of RHS are independent, so each warp takes two of them and runs the whole substitution inside
+// the warp: lane l holds the residuals of the rows at positions l, l+32, ... (NS of them) of its two columns in
+// registers; step j broadcasts y_j = r_j / T_jj from the lane that owns row j by one shuffle and every lane
+// subtracts T_ij y_j from its rows, T read column by column from shared memory (stored transposed, Tt[j][i],
+// zero on and above the diagonal, so no lane needs a predicate and row j keeps its final residual).  A step is
+// one multiply, one shuffle and one multiply-add on the dependent chain and there is no block barrier inside
+// the substitution (the earlier blocked scheme with a barrier per eight rows took 1.8 k cycles per eight rows
+// at C = 48; this one takes about 35 cycles per row).
 // ---------------------------------------------------------------------------
-template <bool BWD>
+inline int team_solve_ns(int C) { return (C + 31) / 32; }
+inline size_t team_solve_smem(int C, int K)
+{
+    const size_t nc = K * K > 32 ? K * K : 32;
+    return sizeof(float) * ((size_t)C * (32 * team_solve_ns(C) + 1) + ((C + 3) & ~3) + (size_t)C * nc + (size_t)C * (nc | 1));
+}
+
+template <bool BWD, int NS>
 __global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict__ w, float* __restrict__ A, int C, int K,
                                                          unsigned char* __restrict__ wop, int NCH, unsigned wbytes,
                                                          float* __restrict__ logdet_out, int HW)
@@ -59,100 +69,108 @@ __global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the wavefront kernel may set itself up meanwhile
     if (logdet_out != nullptr && blockIdx.x == gridDim.x - 1 && threadIdx.x >= 480)
         warp_logdet(w, logdet_out, C, HW, K, threadIdx.x & 31);        // the layer's log-det, by a warp of the lightest CTA
+    constexpr int C32 = 32 * NS, CP = C32 + 1;
     const int KK = K * K, ctr = KK - 1;
-    const int tid = threadIdx.x, NT = blockDim.x;
+    const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = NT >> 5;
     const int b = blockIdx.x;
     const bool ident = b >= C;                // CTAs C, C+1, ...: 32-column chunks of the identity (tap 0)
     const int c0 = ident ? (b - C) * 32 : 0;  // first identity column of this CTA
     const int NC = ident ? min(32, C - c0) : KK;   // right-hand-side columns
-    float* L = sm;                            // [C][C]  L[i][j], j <= i
-    float* invd = sm + C * C;                 // [C]
-    float* RHS = invd + ((C + 3) & ~3);       // [C][NC]  residuals
-    float* Y = RHS + C * (KK > 32 ? KK : 32); // [C][NC]  solved rows
+    const int NCB = KK > 32 ? KK : 32, YS = NCB | 1;
+    float* Tt = sm;                           // [C][CP]   Tt[pa*CP + pi] = T[row at position pi][row at position pa], pi > pa
+    float* invd = Tt + C * CP;                // [C]       1 / T[p][p], by position
+    float* RHS = invd + ((C + 3) & ~3);       // [C][NC]   by row index
+    float* Y = RHS + C * NCB;                 // [C][YS]   solved rows, by row index
+    auto idx = [&](int pos) { return BWD ? C - 1 - pos : pos; };              // position in solve order -> row index
 
-    for (int e0 = tid; e0 < C * C; e0 += NT * 8) {
+    // every global load of the CTA is issued before the first shared-memory store that waits for one
+    const unsigned mKK = 0xFFFFFFFFu / (unsigned)KK + 1u;                      // e / KK = umulhi(e, mKK) for e < 2^16
+    float rv[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const int e = tid + q * NT;
+        rv[q] = 0.f;
+        if (!ident && e < C * KK) {
+            const int m = KK == 1 ? e : (int)__umulhi((unsigned)e, mKK), kk = e - m * KK;
+            rv[q] = BWD ? __ldg(w + (size_t)b * C * KK + e) : __ldg(w + ((size_t)m * C + b) * KK + kk);
+        }
+    }
+    for (int e0 = tid; e0 < C * C32 || e0 == tid; e0 += NT * 8) {            // at least one trip: it also stores rv
         float tv[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-            const int e = e0 + q * NT;
-            tv[q] = (e < C * C) ? __ldg(w + (size_t)e * KK + ctr) : 0.f;
+            const int e = e0 + q * NT, pa = e / C32, pi = e - pa * C32;
+            tv[q] = 0.f;
+            if (e < C * C32 && pi < C && pi >= pa) {
+                const int row = BWD ? idx(pa) : pi, col = BWD ? idx(pi) : pa;   // T[pi][pa] = L[pi][pa] or L^T: L[idx(pa)][idx(pi)]
+                tv[q] = __ldg(w + ((size_t)row * C + col) * KK + ctr);
+            }
+        }
+        if (e0 == tid) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (!ident && tid + q * NT < C * KK) RHS[tid + q * NT] = rv[q];
         }
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-            const int e = e0 + q * NT;
-            if (e < C * C) {
-                const int i = e / C, j = e - i * C;
-                L[e] = (j <= i) ? tv[q] : 0.f;
-                if (i == j) invd[i] = 1.0f / tv[q];
+            const int e = e0 + q * NT, pa = e / C32, pi = e - pa * C32;
+            if (e < C * C32) {
+                Tt[pa * CP + pi] = pi == pa ? 0.f : tv[q];
+                if (pi == pa) invd[pa] = 1.0f / tv[q];
             }
         }
     }
-    if (ident) {
-        for (int e = tid; e < C * NC; e += NT) RHS[e] = (e / NC == c0 + e % NC) ? 1.f : 0.f;
-    } else {
-        for (int e0 = tid; e0 < C * KK; e0 += NT * 4) {
-            float tv[4];
+    if (!ident)
+        for (int e = tid + 8 * NT; e < C * KK; e += NT) {                      // kernels beyond 4096 right-hand-side values
+            const int m = e / KK, kk = e - m * KK;
+            RHS[e] = BWD ? __ldg(w + (size_t)b * C * KK + e) : __ldg(w + ((size_t)m * C + b) * KK + kk);
+        }
+    __syncthreads();
+
+    for (int cb = 2 * warp; cb < NC; cb += 2 * nwarps) {
+        float r[NS][2];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int e = e0 + q * NT;
-                if (e < C * KK) {
-                    const int m = e / KK, kk = e - m * KK;
-                    tv[q] = BWD ? __ldg(w + ((size_t)b * C + m) * KK + kk) : __ldg(w + ((size_t)m * C + b) * KK + kk);
+        for (int s = 0; s < NS; ++s)
+#pragma unroll
+            for (int col = 0; col < 2; ++col) {
+                const int p = lane + 32 * s, c = cb + col;
+                float v = 0.f;
+                if (p < C && c < NC) v = ident ? (idx(p) == c0 + c ? 1.f : 0.f) : RHS[idx(p) * NC + c];
+                r[s][col] = v;
+            }
+#pragma unroll
+        for (int sj = 0; sj < NS; ++sj) {
+            const int jend = min(32, C - 32 * sj);
+#pragma unroll 4
+            for (int jj = 0; jj < jend; ++jj) {
+                const int j = 32 * sj + jj;
+                float t[NS];
+#pragma unroll
+                for (int s = sj; s < NS; ++s) t[s] = Tt[j * CP + lane + 32 * s];
+                const float dj = invd[j];
+#pragma unroll
+                for (int col = 0; col < 2; ++col) {
+                    const float yj = __shfl_sync(0xffffffffu, r[sj][col] * dj, jj);
+#pragma unroll
+                    for (int s = sj; s < NS; ++s) r[s][col] = fmaf(-t[s], yj, r[s][col]);
                 }
             }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int e = e0 + q * NT;
-                if (e < C * KK) RHS[e] = tv[q];
-            }
         }
+#pragma unroll
+        for (int s = 0; s < NS; ++s)
+#pragma unroll
+            for (int col = 0; col < 2; ++col) {
+                const int p = lane + 32 * s, c = cb + col;
+                if (p < C && c < NC) Y[idx(p) * YS + c] = r[s][col] * invd[p];
+            }
     }
     __syncthreads();
-    // thread = (row lane ty, column tx): no divisions inside the substitution loop
-    constexpr int NBK = 8;
-    const int NCP = NC <= 32 ? 32 : NC;
-    const int tx = tid % NCP, ty = tid / NCP, TY = NT / NCP;
-    auto idx = [&](int pos) { return BWD ? C - 1 - pos : pos; };              // position in solve order -> row index
-    auto tval = [&](int pi, int pa) {                                          // T[row at pi][row at pa], pi behind pa
-        const int i = idx(pi), a = idx(pa);
-        return BWD ? L[a * C + i] : L[i * C + a];
-    };
-    for (int b0 = 0; b0 < C; b0 += NBK) {
-        const int nb = min(NBK, C - b0);
-        if (tx < NC && ty < TY) {
-            float rr[NBK], yy[NBK];
-#pragma unroll
-            for (int q = 0; q < NBK; ++q) rr[q] = q < nb ? RHS[idx(b0 + q) * NC + tx] : 0.f;
-#pragma unroll
-            for (int q = 0; q < NBK; ++q) {
-                yy[q] = q < nb ? rr[q] * invd[idx(b0 + (q < nb ? q : 0))] : 0.f;
-#pragma unroll
-                for (int q2 = q + 1; q2 < NBK; ++q2)
-                    if (q2 < nb) rr[q2] = fmaf(-tval(b0 + q2, b0 + q), yy[q], rr[q2]);
-            }
-            if (ty == 0) {
-#pragma unroll
-                for (int q = 0; q < NBK; ++q)
-                    if (q < nb) Y[idx(b0 + q) * NC + tx] = yy[q];
-            }
-            const int nrest = C - (b0 + nb);                                   // rows behind the block
-            for (int ri = ty; ri < nrest; ri += TY) {
-                const int pi = b0 + nb + ri, i = idx(pi);
-                float acc = RHS[i * NC + tx];
-#pragma unroll
-                for (int q = 0; q < NBK; ++q)
-                    if (q < nb) acc = fmaf(-tval(pi, b0 + q), yy[q], acc);
-                RHS[i * NC + tx] = acc;
-            }
-        }
-        __syncthreads();
-    }
+
     if (wop == nullptr) {
-        for (int e = tid; e < C * NC; e += NT) {
-            const int col = e / C, a = e - col * C;               // a fastest: coalesced stores
-            const float v = Y[a * NC + col];
-            if (ident) A[(size_t)(c0 + col) * C + a] = v;         // A[0][b' = c0 + col][a]
-            else if (col != ctr) A[((size_t)(KK - 1 - col) * C + b) * C + a] = v;
+        for (int col = warp; col < NC; col += nwarps) {
+            if (!ident && col == ctr) continue;
+            float* dst = ident ? A + (size_t)(c0 + col) * C : A + ((size_t)(KK - 1 - col) * C + b) * C;   // A[tap][b][.]
+            for (int a = lane; a < C; a += 32) dst[a] = Y[a * YS + col];
         }
         return;
     }
@@ -160,22 +178,49 @@ __global__ void __launch_bounds__(512) team_solve_kernel(const float* __restrict
     //   [dh][chunk % NCH][plane 0,1: tf32 hi | plane 2: bf16 remainder | plane 3: bf16 value][row = dw*C + a][16 bytes],
     // chunk = input channel / 8; the sign is flipped for every tap but tap 0.
     const int KC = K * C;
-    for (int e = tid; e < C * NC; e += NT) {
-        const int col = e / C, a = e - col * C;
+    for (int col = warp; col < NC; col += nwarps) {
         if (!ident && col == ctr) continue;
         const int tap = ident ? 0 : KK - 1 - col, ci = ident ? c0 + col : b;
-        const float v = ident ? Y[a * NC + col] : -Y[a * NC + col];
-        const float hi = tf32_hi(v);
-        const int chunk = ci >> 3, j = ci & 7, r = chunk / NCH, cl = chunk - r * NCH;
-        const int dh = tap / K, dw = tap - dh * K, row = dw * C + a;
-        unsigned char* blk = wop + (size_t)r * wbytes + (size_t)((dh * NCH + cl) * 4) * KC * 16;
-        *reinterpret_cast<float*>(blk + ((size_t)(j >> 2) * KC + row) * 16 + (j & 3) * 4) = hi;
-        *reinterpret_cast<__nv_bfloat16*>(blk + ((size_t)2 * KC + row) * 16 + j * 2) = __float2bfloat16_rn(v - hi);
-        *reinterpret_cast<__nv_bfloat16*>(blk + ((size_t)3 * KC + row) * 16 + j * 2) = __float2bfloat16_rn(v);
+        const int chunk = ci >> 3, j = ci & 7, rk = chunk / NCH, cl = chunk - rk * NCH;
+        const int dh = tap / K, dw = tap - dh * K;
+        unsigned char* blk = wop + (size_t)rk * wbytes + (size_t)((dh * NCH + cl) * 4) * KC * 16;
+        for (int a = lane; a < C; a += 32) {
+            const float y = Y[a * YS + col];
+            const float v = ident ? y : -y;
+            const float hi = tf32_hi(v);
+            const int row = dw * C + a;
+            *reinterpret_cast<float*>(blk + ((size_t)(j >> 2) * KC + row) * 16 + (j & 3) * 4) = hi;
+            *reinterpret_cast<__nv_bfloat16*>(blk + ((size_t)2 * KC + row) * 16 + j * 2) = __float2bfloat16_rn(v - hi);
+            *reinterpret_cast<__nv_bfloat16*>(blk + ((size_t)3 * KC + row) * 16 + j * 2) = __float2bfloat16_rn(v);
+        }
     }
 }
 
-inline size_t team_solve_smem(int C, int K) { return sizeof(float) * ((size_t)C * C + ((C + 3) & ~3) + 2 * (size_t)C * (K * K > 32 ? K * K : 32)); }
+// Launch on `st` (grid: one CTA per input channel plus the identity chunks); cudaSuccess or the launch's error.
+inline cudaError_t team_solve_launch(bool bwd, const float* w, float* A, int C, int K, unsigned char* wop, int NCH,
+                                     unsigned wbytes, float* logdet_out, int HW, cudaStream_t st)
+{
+    using Kern = void (*)(const float*, float*, int, int, unsigned char*, int, unsigned, float*, int);
+    Kern kern = nullptr;
+    switch (team_solve_ns(C) * 2 + (bwd ? 1 : 0)) {
+    case 2: kern = team_solve_kernel<false, 1>; break;
+    case 3: kern = team_solve_kernel<true, 1>; break;
+    case 4: kern = team_solve_kernel<false, 2>; break;
+    case 5: kern = team_solve_kernel<true, 2>; break;
+    case 6: kern = team_solve_kernel<false, 3>; break;
+    case 7: kern = team_solve_kernel<true, 3>; break;
+    case 8: kern = team_solve_kernel<false, 4>; break;
+    case 9: kern = team_solve_kernel<true, 4>; break;
+    default: return cudaErrorInvalidValue;
+    }
+    const size_t sm = team_solve_smem(C, K);
+    if (sm > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+        if (e != cudaSuccess) return e;
+    }
+    kern<<<C + (C + 31) / 32, 512, sm, st>>>(w, A, C, K, wop, NCH, wbytes, logdet_out, HW);
+    return cudaGetLastError();
+}
 
 // ---------------------------------------------------------------------------
 struct TeamParams {

@@ -54,11 +54,10 @@ int tensor_launch(const TensorPlan& pl, bool bwd, const float* rhs, const float*
 {
     if (((reinterpret_cast<uintptr_t>(rhs) | reinterpret_cast<uintptr_t>(out)) & 15) != 0) return INVCONV_UNSUPPORTED;
     {
-        const size_t sm = team_solve_smem(g.C, g.k);
-        auto kern = bwd ? team_solve_kernel<true> : team_solve_kernel<false>;
-        const int rc = set_smem_limit(kern, sm);
-        if (rc) return rc;
-        kern<<<g.C + (g.C + 31) / 32, 512, sm, st>>>(w, A, g.C, g.k, wop, pl.NCH, pl.wbytes, logdet_out, g.H * g.W);
+        if (team_solve_launch(bwd, w, A, g.C, g.k, wop, pl.NCH, pl.wbytes, logdet_out, g.H * g.W, st) != cudaSuccess) {
+            cudaGetLastError();
+            return INVCONV_CUDA_ERROR;
+        }
         const int rl = check_launch();
         if (rl) return rl;
     }
