@@ -7,7 +7,9 @@
 // column offset cannot be a start address here); the row offset dh selects which rows of x are staged.
 //
 // A CTA owns one kernel row dh (its k accumulators [co x ci] live in tensor memory, k*C columns, each fed by
-// its own issuing warp so that an accumulator always receives its products in the same order) and a share
+// one issuing warp -- at most four of them, the first also takes a fifth accumulator -- so that an accumulator
+// always receives its products in the same order; twelve warps leave every scheduler three, which is what lets
+// the producers keep a unit's loads in registers one unit ahead) and a share
 // of the (image, row band) units; per unit the producer warps stage grad_y and the k shifted copies of x
 // (rounded to tf32, single pass: grad_w's tolerance admits it, see the header of the library),
 // double-buffered against the MMA issue.  Partial sums per share go to the workspace; gradw_reduce_kernel
@@ -31,7 +33,7 @@ struct GradWTensorParams {
     unsigned tmem_cols, planeA, planeB, stage_bytes;
 };
 
-__global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorParams p)
+__global__ void __maxnreg__(144) gradw_tensor_kernel(const GradWTensorParams p)
 {
     extern __shared__ __align__(128) unsigned char gsmem[];
     const int tid = threadIdx.x, warp = tid >> 5;
@@ -49,10 +51,11 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
     volatile int* gave_up = reinterpret_cast<volatile int*>(bars + 6);
 
+    const int NIW = K < kGradWTensorIssuers ? K : kGradWTensorIssuers;     // issuing warps
     if (tid == 0) {
         mbar_init(full + 0, 256); mbar_init(full + 1, 256);
-        mbar_init(empty + 0, K); mbar_init(empty + 1, K);
-        mbar_init(done, K);
+        mbar_init(empty + 0, NIW); mbar_init(empty + 1, NIW);
+        mbar_init(done, NIW);
         *gave_up = 0;
         fence_mbar_init();
     }
@@ -97,59 +100,83 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
         }
         const size_t copy_bytes = (size_t)nchunk * planeC;
         const bool shuffle_left = (32 % QW) == 0;          // a row's quads never straddle a warp
+        // four items of unit u: the loads ...
+        auto load4 = [&](int u, int j0, float4 (&a)[4], float4 (&b1)[4]) {
+            const int n = u / p.nbands, r = u - n * p.nbands;
+            const float* gyb = p.gy + (size_t)n * C * HW + (size_t)r * RB * W;        // first row of the band
+            const float* xb = p.x + (size_t)n * C * HW + ((size_t)r * RB - dh) * W;   // ... of the rows dh above it
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                a[j] = b1[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                const int h = r * RB + hl_[j0 + j];
+                if (goff[j0 + j] >= 0 && h < H &&
+                    INVCONV_CHECKED((size_t)n * C * HW + (size_t)r * RB * W + goff[j0 + j] + 3, (size_t)p.B * C * HW, 202)) {
+                    a[j] = __ldg(reinterpret_cast<const float4*>(gyb + goff[j0 + j]));
+                    if (h >= dh) b1[j] = __ldg(reinterpret_cast<const float4*>(xb + goff[j0 + j]));
+                }
+            }
+        };
+        // the quad to the left of each item's quad of x: from the neighbouring lane where a row's quads never
+        // straddle a warp, else loaded (late: widths that are no power of two pay that latency)
+        auto left4 = [&](int u, int j0, const float4 (&b1)[4], float4 (&b0)[4]) {
+            if (shuffle_left) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float4 t;
+                    t.x = __shfl_up_sync(0xffffffffu, b1[j].x, 1); t.y = __shfl_up_sync(0xffffffffu, b1[j].y, 1);
+                    t.z = __shfl_up_sync(0xffffffffu, b1[j].z, 1); t.w = __shfl_up_sync(0xffffffffu, b1[j].w, 1);
+                    b0[j] = left[j0 + j] ? t : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            } else {
+                const int n = u / p.nbands, r = u - n * p.nbands;
+                const float* xb = p.x + (size_t)n * C * HW + ((size_t)r * RB - dh) * W;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    b0[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    const int h = r * RB + hl_[j0 + j];
+                    if (goff[j0 + j] >= 0 && h < H && h >= dh && left[j0 + j]) b0[j] = __ldg(reinterpret_cast<const float4*>(xb + goff[j0 + j] - 4));
+                }
+            }
+        };
+        // ... and the conversions and stores into stage `sa` (grad_y) / `sb` (the K shifted copies of x)
+        auto store4 = [&](int j0, const float4 (&a)[4], const float4 (&b1)[4], const float4 (&b0)[4], unsigned char* sa, unsigned char* sb) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (goff[j0 + j] < 0) continue;
+                if (!INVCONV_CHECKED(soff[j0 + j] + 15, copy_bytes, 201)) continue;
+                unsigned char* da_ = sa + soff[j0 + j];
+                unsigned char* db_ = sb + soff[j0 + j];
+                *reinterpret_cast<float4*>(da_) = make_float4(tf32_hi(a[j].x), tf32_hi(a[j].y), tf32_hi(a[j].z), tf32_hi(a[j].w));
+                const float x0 = tf32_hi(b0[j].x), x1 = tf32_hi(b0[j].y), x2 = tf32_hi(b0[j].z), x3 = tf32_hi(b0[j].w);
+                const float x4 = tf32_hi(b1[j].x), x5 = tf32_hi(b1[j].y), x6 = tf32_hi(b1[j].z), x7 = tf32_hi(b1[j].w);
+                // copy dw holds x[.., w - dw]: elements 4-dw .. 7-dw of the two loaded quads
+                *reinterpret_cast<float4*>(db_) = make_float4(x4, x5, x6, x7);
+                if (K > 1) *reinterpret_cast<float4*>(db_ + copy_bytes) = make_float4(x3, x4, x5, x6);
+                if (K > 2) *reinterpret_cast<float4*>(db_ + 2 * copy_bytes) = make_float4(x2, x3, x4, x5);
+                if (K > 3) *reinterpret_cast<float4*>(db_ + 3 * copy_bytes) = make_float4(x1, x2, x3, x4);
+                if (K > 4) *reinterpret_cast<float4*>(db_ + 4 * copy_bytes) = make_float4(x0, x1, x2, x3);
+            }
+        };
+        // The first four items of a unit are requested one unit ahead, so that their memory latency runs under
+        // the conversions, stores and barrier waits of the unit before (a thread rarely has more than four).
+        float4 na[4], nb1[4];
+        if (share < nunits) load4(share, 0, na, nb1);
         int it = 0;
         for (int u = share; u < nunits; u += p.S, ++it) {
-            const int n = u / p.nbands, r = u - n * p.nbands;
             const int st = it & 1;
+            float4 a[4], b1[4], b0[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { a[j] = na[j]; b1[j] = nb1[j]; }
+            if (u + p.S < nunits) load4(u + p.S, 0, na, nb1);
+            left4(u, 0, b1, b0);
             if (it >= 2) wait_bar(empty + st, ((it >> 1) - 1) & 1);
             unsigned char* sa = gsmem + (size_t)st * p.stage_bytes;
             unsigned char* sb = sa + copy_bytes;
-            const float* gyb = p.gy + (size_t)n * C * HW + (size_t)r * RB * W;        // first row of the band
-            const float* xb = p.x + (size_t)n * C * HW + ((size_t)r * RB - dh) * W;   // ... of the rows dh above it
-            // four items per pass: all loads first, then the conversions and stores
-#pragma unroll
-            for (int j0 = 0; j0 < 8; j0 += 4) {
-                if (j0 * 256 >= items) break;
-                float4 a[4], b1[4], b0[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    a[j] = b1[j] = b0[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    const int h = r * RB + hl_[j0 + j];
-                    if (goff[j0 + j] >= 0 && h < H &&
-                        INVCONV_CHECKED((size_t)n * C * HW + (size_t)r * RB * W + goff[j0 + j] + 3, (size_t)p.B * C * HW, 202)) {
-                        a[j] = __ldg(reinterpret_cast<const float4*>(gyb + goff[j0 + j]));
-                        if (h >= dh) {
-                            b1[j] = __ldg(reinterpret_cast<const float4*>(xb + goff[j0 + j]));
-                            if (left[j0 + j] && !shuffle_left) b0[j] = __ldg(reinterpret_cast<const float4*>(xb + goff[j0 + j] - 4));
-                        }
-                    }
-                }
-                if (shuffle_left) {
-                    // the quad to the left is the previous lane's quad (quads of a row are consecutive lanes)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        float4 t;
-                        t.x = __shfl_up_sync(0xffffffffu, b1[j].x, 1); t.y = __shfl_up_sync(0xffffffffu, b1[j].y, 1);
-                        t.z = __shfl_up_sync(0xffffffffu, b1[j].z, 1); t.w = __shfl_up_sync(0xffffffffu, b1[j].w, 1);
-                        if (left[j0 + j]) b0[j] = t;
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (goff[j0 + j] < 0) continue;
-                    if (!INVCONV_CHECKED(soff[j0 + j] + 15, copy_bytes, 201)) continue;
-                    unsigned char* da_ = sa + soff[j0 + j];
-                    unsigned char* db_ = sb + soff[j0 + j];
-                    *reinterpret_cast<float4*>(da_) = make_float4(tf32_hi(a[j].x), tf32_hi(a[j].y), tf32_hi(a[j].z), tf32_hi(a[j].w));
-                    const float x0 = tf32_hi(b0[j].x), x1 = tf32_hi(b0[j].y), x2 = tf32_hi(b0[j].z), x3 = tf32_hi(b0[j].w);
-                    const float x4 = tf32_hi(b1[j].x), x5 = tf32_hi(b1[j].y), x6 = tf32_hi(b1[j].z), x7 = tf32_hi(b1[j].w);
-                    // copy dw holds x[.., w - dw]: elements 4-dw .. 7-dw of the two loaded quads
-                    *reinterpret_cast<float4*>(db_) = make_float4(x4, x5, x6, x7);
-                    if (K > 1) *reinterpret_cast<float4*>(db_ + copy_bytes) = make_float4(x3, x4, x5, x6);
-                    if (K > 2) *reinterpret_cast<float4*>(db_ + 2 * copy_bytes) = make_float4(x2, x3, x4, x5);
-                    if (K > 3) *reinterpret_cast<float4*>(db_ + 3 * copy_bytes) = make_float4(x1, x2, x3, x4);
-                    if (K > 4) *reinterpret_cast<float4*>(db_ + 4 * copy_bytes) = make_float4(x0, x1, x2, x3);
-                }
+            store4(0, a, b1, b0, sa, sb);
+            if (4 * 256 < items) {
+                load4(u, 4, a, b1);
+                left4(u, 4, b1, b0);
+                store4(4, a, b1, b0, sa, sb);
             }
             fence_proxy_async();
             mbar_arrive(full + st);
@@ -177,11 +204,9 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
             }
             umma::fence_before_sync();
         }
-    } else if ((tid & 31) == 0 && warp - 8 < K) {
-        // ------------------------------------------------ MMA issue: warp 8 + dw owns the accumulator of tap (dh, dw)
-        const int dw = warp - 8;
+    } else if ((tid & 31) == 0 && warp - 8 < NIW) {
+        // ------------------------------------------------ MMA issue: warp 8 + i owns the accumulators of taps (dh, i), (dh, i + NIW)
         const uint32_t idesc = umma::make_idesc(umma::kFmtTF32, (uint32_t)C);
-        const uint32_t dcol = tmem + (uint32_t)(dw * C);
         const uint32_t kstep = 2 * (planeC >> 4), copy = (uint32_t)nchunk * (planeC >> 4);
         int it = 0;
         for (int u = share; u < nunits; u += p.S, ++it) {
@@ -189,11 +214,14 @@ __global__ void __launch_bounds__(512, 1) gradw_tensor_kernel(const GradWTensorP
             wait_bar(full + st, (it >> 1) & 1);
             umma::fence_after_sync();
             const uint32_t sa = smem_u32(gsmem + (size_t)st * p.stage_bytes);
-            uint64_t da = umma::make_desc(sa, planeC);
-            uint64_t db = umma::make_desc(sa + (uint32_t)nchunk * planeC, planeC) + (uint64_t)(dw * copy);
-            for (int ks = 0; ks < p.nk; ++ks) {
-                umma::mma_tf32(dcol, da, db, idesc, (it > 0 || ks > 0) ? 1u : 0u);
-                da += kstep; db += kstep;
+            for (int dw = warp - 8; dw < K; dw += NIW) {
+                const uint32_t dcol = tmem + (uint32_t)(dw * C);
+                uint64_t da = umma::make_desc(sa, planeC);
+                uint64_t db = umma::make_desc(sa + (uint32_t)nchunk * planeC, planeC) + (uint64_t)(dw * copy);
+                for (int ks = 0; ks < p.nk; ++ks) {
+                    umma::mma_tf32(dcol, da, db, idesc, (it > 0 || ks > 0) ? 1u : 0u);
+                    da += kstep; db += kstep;
+                }
             }
             umma::commit(empty + st);
         }

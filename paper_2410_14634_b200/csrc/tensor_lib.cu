@@ -88,7 +88,7 @@ int gradw_tensor_launch(const GradWTensorPlan& pl, const float* gy, const float*
     prm.tmem_cols = pl.tmem_cols; prm.planeA = pl.planeA; prm.planeB = pl.planeB; prm.stage_bytes = pl.stage_bytes;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(pl.grid);
-    cfg.blockDim = dim3(kGradWTensorProducers + 32 * g.k);
+    cfg.blockDim = dim3(kGradWTensorProducers + 32 * (g.k < kGradWTensorIssuers ? g.k : kGradWTensorIssuers));
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

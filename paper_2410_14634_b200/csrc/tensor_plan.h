@@ -65,6 +65,7 @@ struct GradWTensorPlan {
     size_t smem = 0;
 };
 
+constexpr int kGradWTensorIssuers = 4;        // MMA-issuing warps at most (a fifth accumulator shares the first warp)
 constexpr int kGradWTensorProducers = 256;    // warps 0-7 stage the operands (0-3 also write the result); warps 8.. issue the MMAs, one per kernel column
 
 inline GradWTensorPlan plan_gradw_tensor(int B, int C, int H, int W, int K, size_t max_smem, int sms)

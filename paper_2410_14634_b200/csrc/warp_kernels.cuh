@@ -116,6 +116,19 @@ __device__ void build_transformed_kernel(const float* __restrict__ w, float* As)
 {
     constexpr int KK = K * K, CP = ColVec<C>::CP;
     constexpr int ctr = KK - 1;
+    // the taps of this thread's first entry are requested before the centre tap, so that one memory latency
+    // covers both (the entry needs L^-1, which needs the centre tap)
+    float wpre[C];
+    {
+        const int e = threadIdx.x;
+        const int b = (e / C) % C, tap = e / (C * C);
+        const int t = (K - 1 - tap / K) * K + (K - 1 - tap % K);
+#pragma unroll
+        for (int m = 0; m < C; ++m) {
+            wpre[m] = 0.f;
+            if (e < KK * C * C && tap != 0) wpre[m] = BWD ? __ldg(w + (b * C + m) * KK + t) : __ldg(w + (m * C + b) * KK + t);
+        }
+    }
     float L[C][C], Li[C][C];
 #pragma unroll
     for (int i = 0; i < C; ++i)
@@ -155,7 +168,8 @@ __device__ void build_transformed_kernel(const float* __restrict__ w, float* As)
 #pragma unroll
                     for (int j = 0; j < C; ++j)
                         if (i == (BWD ? m : a) && j == (BWD ? a : m)) li = Li[i][j];
-                const float wv = BWD ? __ldg(w + (b * C + m) * KK + t) : __ldg(w + (m * C + b) * KK + t);
+                const float wv = e == (int)threadIdx.x ? wpre[m]
+                                                       : (BWD ? __ldg(w + (b * C + m) * KK + t) : __ldg(w + (m * C + b) * KK + t));
                 v += li * wv;
             }
         }
