@@ -43,6 +43,10 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + ((NW + 31) & ~31));
     float* xs = smem + ((NW + 31) & ~31) + 32 + li * imgf;
 
+    // nothing above touched global memory; x may come from the kernel before this one on the stream.  The next
+    // kernel may be scheduled right away: it waits for this one to complete at its own griddepcontrol.wait.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (has_img && p.bulk && wb == 0 && lane == 0) {
         mbar_init(&bars[li], 1);
         fence_mbar_init();

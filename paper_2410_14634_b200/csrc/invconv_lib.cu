@@ -326,7 +326,19 @@ int launch_masked_conv_ck(const float* x, const float* w, float* y, Geom g, cuda
     prm.x = x; prm.w = w; prm.y = y; prm.B = g.B; prm.H = g.H; prm.W = g.W; prm.ipc = ipc; prm.wpi = wpi;
     const size_t chw = (size_t)g.C * g.H * g.W;
     prm.bulk = ((reinterpret_cast<uintptr_t>(x) & 15) == 0 && chw % 4 == 0) ? 1 : 0;
-    kern<<<(g.B + ipc - 1) / ipc, ipc * wpi * 32, smem, st>>>(prm);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((g.B + ipc - 1) / ipc);
+    cfg.blockDim = dim3(ipc * wpi * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // launch latency overlaps the kernel before
+    attr[0].val.programmaticStreamSerializationAllowed = opt(INVCONV_OPT_DEPENDENT_LAUNCH) ? 1 : 0;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, prm) != cudaSuccess) {
+        cudaGetLastError();
+        return INVCONV_CUDA_ERROR;
+    }
     return check_launch();
 }
 
