@@ -8,6 +8,10 @@
 // loads for C*C*K*K FMAs, and each (channel, row) of y leaves as one coalesced
 // 128-byte store.  The channel mask of the bottom-right tap is applied while the
 // kernel is read.  Bound: HBM (8 bytes per element).
+//
+// Few large images would leave most SMs idle that way, so an image can also be cut into bands of rows, one CTA
+// per band: the band and the K-1 rows above it arrive by one bulk copy per channel (rows of a channel are
+// contiguous), everything else is the same walk.
 #pragma once
 
 #include "common.cuh"
@@ -23,6 +27,8 @@ struct ConvParams {
     int ipc;       // images per CTA
     int wpi;       // warps per image (row bands)
     int bulk;      // images are 16-byte aligned multiples of 16 bytes
+    int bands = 1; // > 1: CTAs per image, each a band of `bh` rows (ipc = 1, bulk copies, W a multiple of 4)
+    int bh = 0;
 };
 
 template <int C, int K>
@@ -32,16 +38,21 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
     constexpr int NW = C * C * K * K;
     constexpr bool WREG = NW <= 108;
     const int H = p.H, W = p.W, HW = H * W, CHW = C * HW;
-    const int imgf = (CHW + 31) & ~31;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int li = warp / p.wpi, wb = warp - li * p.wpi;
-    const int n = blockIdx.x * p.ipc + li;
+    const bool banded = p.bands > 1;
+    const int li = banded ? 0 : warp / p.wpi, wb = banded ? warp : warp - li * p.wpi;
+    const int n = banded ? blockIdx.x / p.bands : blockIdx.x * p.ipc + li;
     const bool has_img = n < p.B;
-    const int band = (H + p.wpi - 1) / p.wpi;
-    const int hb0 = wb * band, hb1 = min(H, hb0 + band);
+    // rows this CTA writes [rb0, rb1) and the first row it holds in shared memory
+    const int rb0 = banded ? (blockIdx.x % p.bands) * p.bh : 0, rb1 = banded ? min(H, rb0 + p.bh) : H;
+    const int rl0 = max(0, rb0 - (K - 1));
+    const int RW = (rb1 - rl0) * W;                                     // floats per channel held in shared memory
+    const int imgf = banded ? 0 : (CHW + 31) & ~31;
+    const int band = (rb1 - rb0 + p.wpi - 1) / p.wpi;
+    const int hb0 = rb0 + wb * band, hb1 = min(rb1, hb0 + band);
     float* ws = smem;                                                   // masked kernel [co][ci][dh][dw]
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + ((NW + 31) & ~31));
-    float* xs = smem + ((NW + 31) & ~31) + 32 + li * imgf;
+    float* xs = smem + ((NW + 31) & ~31) + 32 + li * imgf - rl0 * W;    // xs[ci * RW + row * W + col], row >= rl0
 
     // nothing above touched global memory; x may come from the kernel before this one on the stream.  The next
     // kernel may be scheduled right away: it waits for this one to complete at its own griddepcontrol.wait.
@@ -50,8 +61,14 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
     if (has_img && p.bulk && wb == 0 && lane == 0) {
         mbar_init(&bars[li], 1);
         fence_mbar_init();
-        mbar_expect_tx(&bars[li], (unsigned)CHW * 4u);
-        bulk_g2s(xs, p.x + (size_t)n * CHW, (unsigned)CHW * 4u, &bars[li]);
+        mbar_expect_tx(&bars[li], (unsigned)(C * RW) * 4u);
+        if (banded) {
+#pragma unroll
+            for (int c = 0; c < C; ++c)
+                bulk_g2s(xs + c * RW + rl0 * W, p.x + (size_t)n * CHW + (size_t)c * HW + (size_t)rl0 * W, (unsigned)RW * 4u, &bars[li]);
+        } else {
+            bulk_g2s(xs, p.x + (size_t)n * CHW, (unsigned)CHW * 4u, &bars[li]);
+        }
     }
     if (has_img && !p.bulk) {
         const float* src = p.x + (size_t)n * CHW;
@@ -73,6 +90,7 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
         const bool ok = mbar_wait_bounded(&bars[li], 0);
         if (!__all_sync(0xffffffffu, ok)) { if (lane == 0) raise_status(INVCONV_TIMEOUT); return; }
     }
+    if (hb0 >= hb1) return;                                // a short last band leaves its trailing warps without rows
     float* dst = p.y + (size_t)n * CHW;
     for (int w0 = 0; w0 < W; w0 += 32) {
         const int w = w0 + lane;
@@ -92,7 +110,7 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
 #pragma unroll
                 for (int dw = 0; dw < K; ++dw) {
                     const bool in = row >= 0 && col_ok && w - dw >= 0;
-                    const float t = xs[ci * HW + (in ? row * W + w - dw : 0)];
+                    const float t = xs[ci * RW + (in ? row * W + w - dw : rl0 * W)];
                     xr[(K - q) % K][ci][dw] = in ? t : 0.f;
                 }
         }
@@ -106,7 +124,7 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
 #pragma unroll
                         for (int dw = 0; dw < K; ++dw) {
                             const bool in = col_ok && w - dw >= 0;
-                            const float t = xs[ci * HW + h * W + (in ? w - dw : 0)];      // clamped: no branch
+                            const float t = xs[ci * RW + h * W + (in ? w - dw : 0)];      // clamped: no branch
                             xr[r][ci][dw] = in ? t : 0.f;
                         }
                     float acc[C];
@@ -135,7 +153,7 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
 }
 
 template <int C, int K>
-inline size_t masked_conv_smem(int H, int W, int ipc)
+inline size_t masked_conv_smem(int H, int W, int ipc)      // H: rows held per image (a band plus the K-1 rows above it)
 {
     const size_t imgf = ((size_t)C * H * W + 31) & ~(size_t)31;
     return sizeof(float) * ((((size_t)C * C * K * K + 31) & ~(size_t)31) + 32 + imgf * ipc);

@@ -317,17 +317,35 @@ int launch_masked_conv_ck(const float* x, const float* w, float* y, Geom g, cuda
     if (ipc > g.B) ipc = g.B;
     if (ipc < 1) ipc = 1;
     while (ipc > 1 && masked_conv_smem<C, K>(g.H, g.W, ipc) > kMaxDynSmem) --ipc;
-    const size_t smem = masked_conv_smem<C, K>(g.H, g.W, ipc);
+    size_t smem = masked_conv_smem<C, K>(g.H, g.W, ipc);
+    const size_t chw = (size_t)g.C * g.H * g.W;
+    ConvParams prm;
+    prm.x = x; prm.w = w; prm.y = y; prm.B = g.B; prm.H = g.H; prm.W = g.W;
+    prm.bulk = ((reinterpret_cast<uintptr_t>(x) & 15) == 0 && chw % 4 == 0) ? 1 : 0;
+    int grid = (g.B + ipc - 1) / ipc;
+    // few (fewer CTAs than half the SMs) or very large images: one CTA per band of rows instead, about two CTAs per SM
+    const bool rows_ok = (reinterpret_cast<uintptr_t>(x) & 15) == 0 && g.W % 4 == 0;
+    if (rows_ok && g.H >= 16 && (smem > kMaxDynSmem || 2 * grid <= sm_count())) {
+        int bands = (2 * sm_count() + g.B - 1) / g.B;
+        if (bands > (g.H + 7) / 8) bands = (g.H + 7) / 8;             // at least eight rows per band
+        int bh = (g.H + bands - 1) / bands;
+        while (masked_conv_smem<C, K>(bh + K - 1, g.W, 1) > kMaxDynSmem && bh > 1) bh = (bh + 1) / 2;
+        bands = (g.H + bh - 1) / bh;
+        if (bands > 1 && masked_conv_smem<C, K>(bh + K - 1, g.W, 1) <= kMaxDynSmem) {
+            prm.bands = bands; prm.bh = bh; prm.bulk = 1;
+            ipc = 1;
+            wpi = bh >= 16 ? 4 : (bh >= 8 ? 2 : 1);
+            smem = masked_conv_smem<C, K>(bh + K - 1, g.W, 1);
+            grid = g.B * bands;
+        }
+    }
     if (smem > kMaxDynSmem) return INVCONV_UNSUPPORTED;
     auto kern = masked_conv_warp_kernel<C, K>;
     const int rc = set_smem_limit(kern, smem);
     if (rc) return rc;
-    ConvParams prm;
-    prm.x = x; prm.w = w; prm.y = y; prm.B = g.B; prm.H = g.H; prm.W = g.W; prm.ipc = ipc; prm.wpi = wpi;
-    const size_t chw = (size_t)g.C * g.H * g.W;
-    prm.bulk = ((reinterpret_cast<uintptr_t>(x) & 15) == 0 && chw % 4 == 0) ? 1 : 0;
+    prm.ipc = ipc; prm.wpi = wpi;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((g.B + ipc - 1) / ipc);
+    cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(ipc * wpi * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;

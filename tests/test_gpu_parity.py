@@ -191,6 +191,10 @@ def test_paper_setting_unit_diagonal_one_channel(B, oracle, path):
 
 @pytest.mark.parametrize("path", ["auto", "generic", "team"])
 @pytest.mark.parametrize("shape", [(3, 1, 28, 28, 3), (2, 3, 32, 32, 3), (2, 3, 40, 45, 5), (1, 2, 7, 70, 2), (2, 4, 9, 9, 5),
+                                   # few or large images: one CTA per band of rows (bands that do not divide the
+                                   # height, a one-row last band, images larger than shared memory, widths off 4)
+                                   (2, 3, 64, 64, 5), (1, 1, 256, 256, 5), (3, 2, 40, 36, 3), (1, 4, 100, 20, 2),
+                                   (5, 1, 17, 8, 3), (1, 3, 65, 64, 3), (1, 1, 300, 260, 5), (2, 2, 33, 30, 3), (16, 3, 64, 64, 5),
                                    # tensor-core kernel ("auto" at C = 16..64; "team" keeps the FMA tile kernel): every k
                                    # it serves, bands that do not fill the lanes, ragged last band, wide and 1-pixel-high
                                    # images, more tiles than CTAs, the two 48-channel benchmark shapes
