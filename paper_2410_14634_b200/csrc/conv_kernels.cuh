@@ -36,11 +36,16 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
 {
     extern __shared__ __align__(128) float smem[];
     constexpr int NW = C * C * K * K;
-    constexpr bool WREG = NW <= 108;
+    constexpr bool WREG = NW <= 108;                        // the whole masked kernel fits a lane's registers
+    // otherwise a warp computes one output channel only (its C*K*K weights in registers) and C warps share a band
+    constexpr int CO = WREG ? C : 1;                        // output channels per warp
+    constexpr int NWR = CO * C * K * K;
     const int H = p.H, W = p.W, HW = H * W, CHW = C * HW;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool banded = p.bands > 1;
-    const int li = banded ? 0 : warp / p.wpi, wb = banded ? warp : warp - li * p.wpi;
+    constexpr int WSPLIT = C / CO;                          // warps per band
+    const int bwarp = warp / WSPLIT, co0 = (warp - bwarp * WSPLIT) * CO;
+    const int li = banded ? 0 : bwarp / p.wpi, wb = banded ? bwarp : bwarp - li * p.wpi;
     const int n = banded ? blockIdx.x / p.bands : blockIdx.x * p.ipc + li;
     const bool has_img = n < p.B;
     // rows this CTA writes [rb0, rb1) and the first row it holds in shared memory
@@ -58,7 +63,7 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
     // kernel may be scheduled right away: it waits for this one to complete at its own griddepcontrol.wait.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (has_img && p.bulk && wb == 0 && lane == 0) {
+    if (has_img && p.bulk && wb == 0 && co0 == 0 && lane == 0) {
         mbar_init(&bars[li], 1);
         fence_mbar_init();
         mbar_expect_tx(&bars[li], (unsigned)(C * RW) * 4u);
@@ -72,7 +77,7 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
     }
     if (has_img && !p.bulk) {
         const float* src = p.x + (size_t)n * CHW;
-        for (int i = wb * 32 + lane; i < CHW; i += p.wpi * 32) xs[i] = __ldg(src + i);
+        for (int i = (wb * WSPLIT + co0 / CO) * 32 + lane; i < CHW; i += p.wpi * WSPLIT * 32) xs[i] = __ldg(src + i);
     }
     for (int e = threadIdx.x; e < NW; e += blockDim.x) {
         const int dw = e % K, dh = (e / K) % K, ci = (e / (K * K)) % C, co = e / (K * K * C);
@@ -81,11 +86,9 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
     }
     __syncthreads();
     if (!has_img) return;
-    float wr[WREG ? NW : 1];
-    if constexpr (WREG) {
+    float wr[NWR];
 #pragma unroll
-        for (int e = 0; e < NW; ++e) wr[e] = ws[e];
-    }
+    for (int e = 0; e < NWR; ++e) wr[e] = ws[co0 * C * K * K + e];
     if (p.bulk) {
         const bool ok = mbar_wait_bounded(&bars[li], 0);
         if (!__all_sync(0xffffffffu, ok)) { if (lane == 0) raise_status(INVCONV_TIMEOUT); return; }
@@ -127,24 +130,21 @@ __global__ void __launch_bounds__(256) masked_conv_warp_kernel(ConvParams p)
                             const float t = xs[ci * RW + h * W + (in ? w - dw : 0)];      // clamped: no branch
                             xr[r][ci][dw] = in ? t : 0.f;
                         }
-                    float acc[C];
+                    float acc[CO];
 #pragma unroll
-                    for (int co = 0; co < C; ++co) acc[co] = 0.f;
+                    for (int co = 0; co < CO; ++co) acc[co] = 0.f;
 #pragma unroll
-                    for (int co = 0; co < C; ++co)
+                    for (int co = 0; co < CO; ++co)
 #pragma unroll
                         for (int ci = 0; ci < C; ++ci)
 #pragma unroll
                             for (int dh = 0; dh < K; ++dh)
 #pragma unroll
-                                for (int dw = 0; dw < K; ++dw) {
-                                    const int e = ((co * C + ci) * K + dh) * K + dw;
-                                    const float wv = WREG ? wr[WREG ? e : 0] : ws[e];
-                                    acc[co] = fmaf(wv, xr[(r - dh + K) % K][ci][dw], acc[co]);
-                                }
+                                for (int dw = 0; dw < K; ++dw)
+                                    acc[co] = fmaf(wr[((co * C + ci) * K + dh) * K + dw], xr[(r - dh + K) % K][ci][dw], acc[co]);
                     if (col_ok) {
 #pragma unroll
-                        for (int co = 0; co < C; ++co) dst[co * HW + h * W + w] = acc[co];
+                        for (int co = 0; co < CO; ++co) dst[(co0 + co) * HW + h * W + w] = acc[co];
                     }
                 }
             }

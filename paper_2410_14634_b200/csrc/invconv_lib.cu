@@ -310,10 +310,13 @@ size_t warp_workspace_bytes(int B, int C, int H, int W, int k)
 template <int C, int K>
 int launch_masked_conv_ck(const float* x, const float* w, float* y, Geom g, cudaStream_t st)
 {
+    // warps per band of rows: one, or one per output channel where the kernel does not fit a lane's registers
+    constexpr int wsplit = (C * C * K * K <= 108) ? 1 : C;
+    constexpr int maxw = 8 / wsplit;             // eight warps per CTA
     int wpi = (g.H + 7) / 8;                     // about eight rows per warp
-    if (wpi > 8) wpi = 8;
+    if (wpi > maxw) wpi = maxw;
     if (wpi < 1) wpi = 1;
-    int ipc = 8 / wpi;
+    int ipc = maxw / wpi;
     if (ipc > g.B) ipc = g.B;
     if (ipc < 1) ipc = 1;
     while (ipc > 1 && masked_conv_smem<C, K>(g.H, g.W, ipc) > kMaxDynSmem) --ipc;
@@ -335,6 +338,7 @@ int launch_masked_conv_ck(const float* x, const float* w, float* y, Geom g, cuda
             prm.bands = bands; prm.bh = bh; prm.bulk = 1;
             ipc = 1;
             wpi = bh >= 16 ? 4 : (bh >= 8 ? 2 : 1);
+            if (wpi > maxw) wpi = maxw;
             smem = masked_conv_smem<C, K>(bh + K - 1, g.W, 1);
             grid = g.B * bands;
         }
@@ -346,7 +350,7 @@ int launch_masked_conv_ck(const float* x, const float* w, float* y, Geom g, cuda
     prm.ipc = ipc; prm.wpi = wpi;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(ipc * wpi * 32);
+    cfg.blockDim = dim3(ipc * wpi * wsplit * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
