@@ -73,12 +73,20 @@ inline GradWTensorPlan plan_gradw_tensor(int B, int C, int H, int W, int K, size
     GradWTensorPlan pl;
     if (C % 16 != 0 || C < 16 || C > 128 || K * C > 512 || B < 1 || K > 5 || W % 4 != 0) return pl;
     pl.Wp = W;
-    for (pl.RB = H >= 4 ? 4 : 2; pl.RB >= 2; pl.RB -= 2) {
+    // Rows per unit: four, or more where few channels leave room (a unit then carries a thread's full four
+    // items, and its fixed cost -- one L2 round trip, barrier hand-offs -- is paid less often), as long as every
+    // CTA still gets at least two units to double-buffer.
+    const int cand[4] = {16, 8, 4, 2};
+    pl.RB = 0;
+    for (int i = 0; i < 4; ++i) {
+        const int rb = cand[i];
+        if (rb > 4 && (rb > H || C * rb * (W / 4) > 4 * kGradWTensorProducers || (long long)B * ((H + rb - 1) / rb) < 2LL * (sms / K))) continue;
+        if (rb == 4 && H < 4) continue;
         // one stage: grad_y and K shifted copies of x, [quad][channel][4 pixels] each, plus room for the rows
         // C..127 that the MMA reads (and ignores) behind the last quad plane
-        pl.stage_bytes = (unsigned)(((size_t)(K + 1) * (pl.RB * W / 4) * (C + 1) * 16 + 128 * 16 + 127) & ~(size_t)127);
+        pl.stage_bytes = (unsigned)(((size_t)(K + 1) * (rb * W / 4) * (C + 1) * 16 + 128 * 16 + 127) & ~(size_t)127);
         pl.smem = 2 * (size_t)pl.stage_bytes + 256;
-        if (pl.smem <= max_smem) break;
+        if (pl.smem <= max_smem) { pl.RB = rb; break; }
     }
     if (pl.RB < 2 || (pl.RB * W) % 8 != 0 || C * pl.RB * (W / 4) > 8 * kGradWTensorProducers) return pl;
     pl.nbands = (H + pl.RB - 1) / pl.RB;
