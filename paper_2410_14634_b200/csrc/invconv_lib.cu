@@ -895,7 +895,7 @@ __global__ void narrow_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* 
         for (size_t u = (size_t)blockIdx.x * blockDim.x + threadIdx.x; u < n / 8; u += stride) {
             const float4 a = reinterpret_cast<const float4*>(in)[2 * u], b = reinterpret_cast<const float4*>(in)[2 * u + 1];
             reinterpret_cast<uint4*>(out)[u] =
-                make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+                make_uint4(pack2_bf16(a.x, a.y), pack2_bf16(a.z, a.w), pack2_bf16(b.x, b.y), pack2_bf16(b.z, b.w));
         }
     } else {
         for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) out[i] = __float2bfloat16_rn(in[i]);

@@ -918,7 +918,7 @@ __device__ __forceinline__ void widen_bf16_warp(float* region, float* second, in
     }
 }
 
-__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
+__device__ __forceinline__ unsigned pack2_bf16(float lo, float hi)
 {
     const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);     // .x = lo in the low half
     return *reinterpret_cast<const unsigned*>(&t);
@@ -1066,7 +1066,7 @@ __global__ void __launch_bounds__(256) warp_wavefront_kernel(WarpParams p)
         const float4* s4 = reinterpret_cast<const float4*>(img);
         for (int u = j * 32 + lane; u < (CHW >> 3); u += p.nb * 32) {
             const float4 a = s4[2 * u], b = s4[2 * u + 1];
-            d16[u] = make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+            d16[u] = make_uint4(pack2_bf16(a.x, a.y), pack2_bf16(a.z, a.w), pack2_bf16(b.x, b.y), pack2_bf16(b.z, b.w));
         }
     }
     if (!GLB && has_img && !narrow) {
