@@ -539,7 +539,9 @@ int launch_gradw(const float* gy, const float* x, float* gw, Geom g, void* ws, c
     // tensor pipe (TF32 inputs) where the fragments line up: rows of whole 8-pixel chunks, conflict-free planes
     // (measured, kernel + reduction: 31 / 58 us against 41 / 87 us for the FMA kernel on the 48-channel shapes,
     // k = 3 / 5; 19 us against 25 us on the 12-channel one with all taps in one CTA)
-    const bool mma = g.W % 8 == 0 && gp.plane % 32 == 4 && opt(INVCONV_OPT_GRADW_TENSOR_PIPE) != 0;
+    // Not below 8 channels: with a handful of entries none of them is large against the cancellation in its own sum,
+    // and TF32 rounding (2^-11 per operand) then shows at 1e-3 of the entry (seen at C = 1, 2 with k = 1).
+    const bool mma = g.C >= 8 && g.W % 8 == 0 && gp.plane % 32 == 4 && opt(INVCONV_OPT_GRADW_TENSOR_PIPE) != 0;
     int shares = gp.nbc;
     if (mma && gp.TC == 1) {                 // tiles of 16 channels: one CTA covers all taps, its own share count
         shares = gp.nbc_all;

@@ -122,6 +122,21 @@ def test_edge_shapes(B, oracle, shape, path):
     check_all(B, oracle, w, y, gx, path)
 
 
+@pytest.mark.parametrize("shape", [(18, 1, 25, 32, 1), (18, 2, 25, 32, 1), (6, 4, 16, 16, 1), (9, 5, 8, 16, 3)], ids=lambda s: "x".join(map(str, s)))
+def test_grad_w_of_few_channels_keeps_fp32_accuracy_under_cancellation(B, oracle, shape):
+    """Few entries in grad_w, each a long sum with heavy cancellation (sum of |terms| about 100 times the sum):
+    operands rounded to TF32 would show at 1e-3 of the entry, so these shapes must stay on fp32 multiply-adds."""
+    import torch
+    Bn, C, H, W, k = shape
+    for seed in range(6):
+        w, y, gx = workloads.make_custom(seed, Bn, C, H, W, k, sigma=0.05)
+        x_ref = oracle.invconv_forward(y, w)
+        _, gw_ref = oracle.invconv_backward(gx, x_ref, w)
+        _, gw = B.invconv_backward(dev(gx), dev(x_ref.astype(np.float32)), dev(w))
+        torch.cuda.synchronize()
+        assert nmax_err(gw.cpu().numpy(), gw_ref) <= 2e-5, seed
+
+
 GW_SEPARATE = [  # shapes for the pixel-parallel grad_w kernel: ragged widths, bands with and without halo rows,
     # more (image, band) items than CTAs, a single pixel, every (C, k) the few-channel family serves
     (1, 1, 1, 1, 2), (3, 1, 28, 28, 3), (2, 3, 32, 32, 3), (1, 3, 64, 64, 5), (2, 4, 9, 11, 5), (1, 2, 7, 9, 5),
