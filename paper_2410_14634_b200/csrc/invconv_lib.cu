@@ -771,8 +771,12 @@ int launch_forward(int path, const float* y, const float* w, float* x, Geom g,
         // buffers off a 16-byte boundary cannot use the bulk copies of the tensor family: the team family serves
         // them from the same workspace (its layout is a prefix of the tensor family's)
         const bool aligned = ((reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(x)) & 15) == 0;
-        if (!aligned && g_forced_path.load() == INVCONV_PATH_AUTO && team_plan(g.B, g.C, g.H, g.W, g.k).ok)
-            return launch_team(false, y, w, x, g, ws, st, logdet_out);
+        if (!aligned && g_forced_path.load() == INVCONV_PATH_AUTO) {
+            if (team_plan(g.B, g.C, g.H, g.W, g.k).ok) return launch_team(false, y, w, x, g, ws, st, logdet_out);
+            generic_wavefront_kernel<false><<<g.B, 256, 0, st>>>(y, w, x, g);      // neither family takes them: the generic one does
+            const int rc = check_launch();
+            return rc ? rc : separate_logdet();
+        }
         return launch_tensor(false, y, w, x, g, ws, st, logdet_out);
     }
     default:
@@ -816,9 +820,17 @@ int launch_backward(int path, const float* gx, const float* x, const float* w, f
     case INVCONV_PATH_TENSOR: {
         if (g.B > 0) {
             const bool aligned = ((reinterpret_cast<uintptr_t>(gx) | reinterpret_cast<uintptr_t>(gy)) & 15) == 0;
-            const int rc = (!aligned && g_forced_path.load() == INVCONV_PATH_AUTO && team_plan(g.B, g.C, g.H, g.W, g.k).ok)
-                               ? launch_team(true, gx, w, gy, g, ws, st)
-                               : launch_tensor(true, gx, w, gy, g, ws, st);
+            int rc;
+            if (!aligned && g_forced_path.load() == INVCONV_PATH_AUTO) {
+                if (team_plan(g.B, g.C, g.H, g.W, g.k).ok) {
+                    rc = launch_team(true, gx, w, gy, g, ws, st);
+                } else {
+                    generic_wavefront_kernel<true><<<g.B, 256, 0, st>>>(gx, w, gy, g);
+                    rc = check_launch();
+                }
+            } else {
+                rc = launch_tensor(true, gx, w, gy, g, ws, st);
+            }
             if (rc) return rc;
         }
         if (gw) return launch_gradw_tensor(gy, x, gw, g, ws, tensor_gradw_offset(g.B, g.C, g.H, g.W, g.k), st, ld);

@@ -339,7 +339,7 @@ def test_a_bounded_wait_that_runs_out_is_reported_once_and_the_context_stays_usa
     assert nmax_err(x.cpu().numpy(), oracle.invconv_forward(y, w)) <= TOL_X
 
 
-@pytest.mark.parametrize("shape", [(3, 16, 8, 8, 3), (9, 48, 16, 16, 3)], ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("shape", [(3, 16, 8, 8, 3), (9, 48, 16, 16, 3), (3, 64, 16, 24, 3), (7, 64, 15, 24, 2)], ids=lambda s: "x".join(map(str, s)))
 def test_unaligned_buffers_on_shapes_of_the_tensor_family(B, oracle, shape):
     """Buffers 4 bytes off a 16-byte boundary: the automatic choice must still serve the shape (the tensor family's
     bulk copies need aligned slices, so another family takes over), forward, backward and masked convolution."""
