@@ -34,7 +34,7 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, one launch, from the ncu captures
 # summarised under profiles/ (per workload; None where no capture exists)
-NCU_TRAFFIC_BYTES = {"mnist": 1.655e6, "wide48_k5": 3.65e6 + 6.33e6}   # wide48_k5: transposed solve + grad_w (profiles/tensor_wavefront_wide48_k5.md)
+NCU_TRAFFIC_BYTES = {"mnist": 1.655e6, "wide48_k5": 3.65e6 + 6.34e6}   # wide48_k5: transposed solve + grad_w (profiles/tensor_wavefront_wide48_k5.md)
 
 METRIC = "invconv_fwd_bwd_images_per_sec"
 UNIT = "images/s"
