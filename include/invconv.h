@@ -83,10 +83,11 @@ int invconv_forward(const float* y, const float* w, float* x,
  *   grad_y [B,C,H,W] out, grad_w [C,C,k,k] out.  grad_w may be NULL (skip it);
  *   grad_y must be non-NULL (grad_w is computed from it).
  * Precision: the solves accumulate in fp32 throughout (the tensor-core family splits every operand into a
- * tf32 part and a bf16 remainder, so its products carry about 19 bits).  For C >= 12 the sum over pixels of
- * grad_w runs on the tensor pipe with its two operands rounded to tf32 (10-bit mantissa) and fp32
- * accumulation: each entry is then accurate to about 3e-4 of the LARGEST entry of grad_w, not of itself;
- * INVCONV_OPT_GRADW_TENSOR_PIPE = 0 selects the fp32 kernel instead. */
+ * tf32 part and a bf16 remainder, so its products carry about 19 bits).  For C >= 8 outside the warp-shuffle
+ * family the sum over pixels of grad_w may run on the tensor pipe with its two operands rounded to tf32
+ * (10-bit mantissa) and fp32 accumulation: each entry is then accurate to about 3e-4 of the LARGEST entry of
+ * grad_w, not of itself; INVCONV_OPT_GRADW_TENSOR_PIPE = 0 selects the fp32 kernel instead.  Below 8 channels
+ * grad_w is always summed from fp32 products. */
 int invconv_backward(const float* grad_x, const float* x, const float* w,
                      float* grad_y, float* grad_w,
                      int B, int C, int H, int W, int k, void* stream);
