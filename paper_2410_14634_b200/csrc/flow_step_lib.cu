@@ -120,9 +120,9 @@ __global__ void __launch_bounds__(256) flow_mix_grad_final_kernel(const float* _
     float* G = fsm;                   // [C*C + C]
     const int NE = C * C + C;
     for (int e = threadIdx.x; e < NE; e += blockDim.x) {
-        float a = 0.f;
-        for (int sh = 0; sh < shares; ++sh) a += __ldcg(partials + (size_t)sh * NE + e);
-        G[e] = a;
+        double a = 0.0;                               // the shares' sums cancel heavily where C is small: add them in double
+        for (int sh = 0; sh < shares; ++sh) a += (double)__ldcg(partials + (size_t)sh * NE + e);
+        G[e] = (float)a;
     }
     __syncthreads();
     for (int e = threadIdx.x; e < C * C; e += blockDim.x) {

@@ -24,8 +24,8 @@ int sm_count();
 template <typename Kern>
 inline int set_smem_limit(Kern kern, size_t smem)
 {
-    // the 48 KB a kernel may use without opting in include its static shared memory (a few words in some kernels)
-    if (smem <= 47 * 1024) return INVCONV_OK;
+    // the 48 KB a kernel may use without opting in include its static shared memory (up to a few KB in some kernels)
+    if (smem <= 40 * 1024) return INVCONV_OK;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
         cudaGetLastError();
         return INVCONV_CUDA_ERROR;

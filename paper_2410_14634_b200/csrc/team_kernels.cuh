@@ -214,7 +214,7 @@ inline cudaError_t team_solve_launch(bool bwd, const float* w, float* A, int C, 
     default: return cudaErrorInvalidValue;
     }
     const size_t sm = team_solve_smem(C, K);
-    if (sm > 47 * 1024) {      // static shared memory counts towards the 48 KB available without opting in
+    if (sm > 40 * 1024) {      // static shared memory counts towards the 48 KB available without opting in
         const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
         if (e != cudaSuccess) return e;
     }

@@ -110,7 +110,7 @@ EDGE = [  # (B, C, H, W, k)
     (9, 16, 16, 16, 3), (3, 32, 8, 8, 5), (17, 48, 16, 4, 2), (5, 64, 12, 16, 4), (1, 48, 16, 16, 5),
     (20, 16, 7, 12, 5), (2, 32, 16, 32, 3), (200, 16, 4, 4, 3), (33, 48, 2, 2, 3), (4, 64, 16, 16, 5),
     # dynamic shared memory of exactly 48 KB beside a kernel's static words (needs the opt-in all the same)
-    (6, 2, 37, 39, 5),
+    (6, 2, 37, 39, 5), (3, 2, 160, 114, 5),
     # kernel transform: more than 4096 right-hand-side values per input channel, four row slots per lane, one channel
     (1, 96, 4, 4, 7), (1, 128, 3, 3, 7), (2, 128, 4, 4, 3), (1, 100, 4, 4, 2), (2, 5, 8, 8, 1), (1, 40, 6, 6, 9),
 ]
