@@ -64,16 +64,21 @@ __global__ void __launch_bounds__(256) flow_mix_kernel(const float* __restrict__
 
 // Partial sums over a share of the (image, pixel tile) items:
 //   G1[o][c] = sum grad_u[n][o][p] * x[n][c][p],   g0[o] = sum grad_u[n][o][p]
-// partials[share][C*C + C].  Thread (o, c-lane) walks the pixels of a staged tile.
+// partials[share][C*C + C] (double).  Thread (o, c-lane) walks the pixels of a staged tile.  With few channels there are
+// few entries, each one long sum that may cancel almost completely (and nothing larger to be measured against), so a
+// thread that owns at most four entries adds the exact fp32 products in double; with many channels the sums
+// stay fp32 (up to 68 per thread).
 __global__ void __launch_bounds__(256) flow_mix_grad_kernel(const float* __restrict__ gu, const float* __restrict__ x,
-                                                            float* __restrict__ partials, int B, int C, int HW, int tiles)
+                                                            double* __restrict__ partials, int B, int C, int HW, int tiles)
 {
     extern __shared__ __align__(16) float fsm[];
     float* tg = fsm;                              // [C][kMixPixels + 1]
     float* tx = tg + C * (kMixPixels + 1);        // [C][kMixPixels + 1]
     const int items = B * tiles, NE = C * C + C;
     const int per = (NE + blockDim.x - 1) / blockDim.x;     // entries per thread (at most 65 for C = 128)
+    const bool wide_acc = per <= 4;
     float acc[68];
+    double dacc[4] = {0.0, 0.0, 0.0, 0.0};
     for (int q = 0; q < 68; ++q) acc[q] = 0.f;
     for (int it = blockIdx.x; it < items; it += gridDim.x) {
         const int n = it / tiles, t0 = (it - n * tiles) * kMixPixels;
@@ -87,6 +92,25 @@ __global__ void __launch_bounds__(256) flow_mix_grad_kernel(const float* __restr
             tx[c * (kMixPixels + 1) + p] = p < np ? __ldg(sx + (size_t)c * HW + p) : 0.f;
         }
         __syncthreads();
+        if (wide_acc) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int e = threadIdx.x + q * blockDim.x;
+                if (q >= per || e >= NE) break;
+                double a = dacc[q];
+                if (e < C * C) {
+                    const int o = e / C, c = e - o * C;
+                    const float* pg = tg + o * (kMixPixels + 1);
+                    const float* px = tx + c * (kMixPixels + 1);
+                    for (int p = 0; p < kMixPixels; ++p) a = fma((double)pg[p], (double)px[p], a);
+                } else {
+                    const float* pg = tg + (e - C * C) * (kMixPixels + 1);
+                    for (int p = 0; p < kMixPixels; ++p) a += (double)pg[p];
+                }
+                dacc[q] = a;
+            }
+            continue;
+        }
         for (int q = 0; q < per; ++q) {
             const int e = threadIdx.x + q * blockDim.x;
             if (e >= NE) break;
@@ -105,39 +129,39 @@ __global__ void __launch_bounds__(256) flow_mix_grad_kernel(const float* __restr
     }
     for (int q = 0; q < per; ++q) {
         const int e = threadIdx.x + q * blockDim.x;
-        if (e < NE) partials[(size_t)blockIdx.x * NE + e] = acc[q];
+        if (e < NE) partials[(size_t)blockIdx.x * NE + e] = wide_acc ? dacc[q < 4 ? q : 0] : (double)acc[q];
     }
 }
 
 // Sums the shares in order and forms the parameter gradients:
 //   grad_V[o][c] = s[c] * G1[o][c] + b[c] * g0[o];  grad_s[c] = sum_o V[o][c] * G1[o][c];  grad_b[c] = sum_o V[o][c] * g0[o].
-__global__ void __launch_bounds__(256) flow_mix_grad_final_kernel(const float* __restrict__ partials, int shares,
+__global__ void __launch_bounds__(256) flow_mix_grad_final_kernel(const double* __restrict__ partials, int shares,
                                                                   const float* __restrict__ V, const float* __restrict__ s,
                                                                   const float* __restrict__ b, float* __restrict__ grad_V,
                                                                   float* __restrict__ grad_s, float* __restrict__ grad_b, int C)
 {
-    extern __shared__ __align__(16) float fsm[];
-    float* G = fsm;                   // [C*C + C]
+    extern __shared__ __align__(16) double fsmd[];
+    double* G = fsmd;                 // [C*C + C]
     const int NE = C * C + C;
     for (int e = threadIdx.x; e < NE; e += blockDim.x) {
-        double a = 0.0;                               // the shares' sums cancel heavily where C is small: add them in double
-        for (int sh = 0; sh < shares; ++sh) a += (double)__ldcg(partials + (size_t)sh * NE + e);
-        G[e] = (float)a;
+        double a = 0.0;
+        for (int sh = 0; sh < shares; ++sh) a += __ldcg(partials + (size_t)sh * NE + e);
+        G[e] = a;
     }
     __syncthreads();
     for (int e = threadIdx.x; e < C * C; e += blockDim.x) {
         const int o = e / C, c = e - o * C;
-        grad_V[e] = fmaf(__ldg(s + c), G[e], __ldg(b + c) * G[C * C + o]);
+        grad_V[e] = (float)((double)__ldg(s + c) * G[e] + (double)__ldg(b + c) * G[C * C + o]);
     }
     for (int c = threadIdx.x; c < C; c += blockDim.x) {
-        float gs = 0.f, gb = 0.f;
+        double gs = 0.0, gb = 0.0;
         for (int o = 0; o < C; ++o) {
-            const float v = __ldg(V + o * C + c);
-            gs = fmaf(v, G[o * C + c], gs);
-            gb = fmaf(v, G[C * C + o], gb);
+            const double v = (double)__ldg(V + o * C + c);
+            gs += v * G[o * C + c];
+            gb += v * G[C * C + o];
         }
-        grad_s[c] = gs;
-        grad_b[c] = gb;
+        grad_s[c] = (float)gs;
+        grad_b[c] = (float)gb;
     }
 }
 
@@ -292,13 +316,13 @@ int invconv_flow_step_backward(const float* grad_u, const float* x, const float*
     if (shares > B * tiles) shares = B * tiles;
     if (shares < 1) shares = 1;
     const size_t NE = (size_t)C * C + C;
-    const size_t part = up256(sizeof(float) * NE * shares);
+    const size_t part = up256(sizeof(double) * NE * shares);
     Scratch sc;
     const int ra = sc.acquire(need + act + part, st);
     if (ra) return ra;
     char* base = static_cast<char*>(sc.p);
     float* grad_x = reinterpret_cast<float*>(base + need);
-    float* partials = reinterpret_cast<float*>(base + need + act);
+    double* partials = reinterpret_cast<double*>(base + need + act);
     int rc = INVCONV_OK;
     if (B > 0) {
         rc = invconv_internal::warp_step_backward(grad_u, x, w, s, V, grad_y, grad_w, Geom{B, C, H, W, k}, sc.p, st);
@@ -320,7 +344,7 @@ int invconv_flow_step_backward(const float* grad_u, const float* x, const float*
         if (rc) return rc;
         shares = 0;
     }
-    const size_t smf = sizeof(float) * NE;
+    const size_t smf = sizeof(double) * NE;
     auto kf = flow_mix_grad_final_kernel;
     rc = invconv_internal::set_smem_limit(kf, smf);
     if (rc) return rc;
