@@ -61,3 +61,48 @@ def test_random_shape_matches_oracle(case):
     gy16_ref, gw16_ref = oracle.invconv_backward(gx16.double().cpu().numpy(), x16.double().cpu().numpy(), w)
     assert stored_ok(gy16, gy16_ref)
     assert nmax_err(gw16.cpu().numpy(), gw16_ref) <= 1e-3
+
+
+@pytest.mark.parametrize("case", sample(77, 80), ids=lambda c: "x".join(map(str, c[1:])))
+def test_random_shape_stays_inside_its_buffers(case):
+    """The caller-workspace forms on buffers with guard regions on both sides: the workspace of exactly the size the
+    library asks for, every output, and the control words (left zero) -- nothing outside them may change."""
+    import torch
+    from paper_2410_14634_b200 import binding
+    seed, B, C, H, W, k = case
+    L = binding.lib()
+    G = 4096
+
+    def guarded(numel, dtype, fill):
+        buf = torch.full((numel + 2 * G,), fill, dtype=dtype, device="cuda")
+        return buf, buf[G:G + numel]
+
+    def intact(buf, numel, fill):
+        return bool((buf[:G] == fill).all()) and bool((buf[G + numel:] == fill).all())
+
+    w, y, gx = workloads.make_custom(seed, B, C, H, W, k, sigma=0.05 / np.sqrt(C))
+    wd, yd, gxd = (torch.from_numpy(a).cuda() for a in (w, y, gx))
+    y16, gx16 = yd.to(torch.bfloat16), gxd.to(torch.bfloat16)
+    ne, nw, dims = y.size, w.size, (B, C, H, W, k)
+    need = max(int(L.invconv_workspace_bytes(*dims)), 256)
+    need16 = max(int(L.invconv_bf16_workspace_bytes(*dims)), 256)
+    wsb, ws = guarded(need, torch.uint8, 0xAB)
+    wsb16, ws16 = guarded(need16, torch.uint8, 0xAB)
+    ws[:256] = 0
+    ws16[:256] = 0
+    outs = {name: guarded(n, dt, 7.0) for name, n, dt in
+            [("x", ne, torch.float32), ("gy", ne, torch.float32), ("f", ne, torch.float32), ("gw", nw, torch.float32),
+             ("x16", ne, torch.bfloat16), ("gy16", ne, torch.bfloat16), ("gw16", nw, torch.float32)]}
+    p = {name: v[1].data_ptr() for name, v in outs.items()}
+    rcs = [L.invconv_forward_ws(yd.data_ptr(), wd.data_ptr(), p["x"], *dims, ws.data_ptr(), need, None),
+           L.invconv_backward_ws(gxd.data_ptr(), p["x"], wd.data_ptr(), p["gy"], p["gw"], *dims, ws.data_ptr(), need, None),
+           L.masked_conv_forward(p["x"], wd.data_ptr(), p["f"], *dims, None),
+           L.invconv_forward_bf16_ws(y16.data_ptr(), wd.data_ptr(), p["x16"], *dims, ws16.data_ptr(), need16, None),
+           L.invconv_backward_bf16_ws(gx16.data_ptr(), p["x16"], wd.data_ptr(), p["gy16"], p["gw16"], *dims, ws16.data_ptr(), need16, None)]
+    torch.cuda.synchronize()
+    assert rcs == [0] * 5 and binding.invconv_get_status() == 0
+    assert intact(wsb, need, 0xAB) and intact(wsb16, need16, 0xAB)
+    assert bool((ws[:256] == 0).all()) and bool((ws16[:256] == 0).all())
+    for name, (buf, view) in outs.items():
+        assert intact(buf, view.numel(), 7.0), name
+        assert bool(torch.isfinite(view.float()).all()), name
