@@ -106,3 +106,69 @@ def test_random_shape_stays_inside_its_buffers(case):
     for name, (buf, view) in outs.items():
         assert intact(buf, view.numel(), 7.0), name
         assert bool(torch.isfinite(view.float()).all()), name
+
+
+def forced_sample(seed, count):
+    rng = np.random.default_rng(seed)
+    out = []
+    for case in sample(seed + 1, count):
+        opts = {"ring": int(rng.integers(0, 2)), "split": int(rng.integers(0, 2)), "pipe": int(rng.integers(0, 2)),
+                "pdl": int(rng.integers(0, 2)), "separate": int(rng.integers(-1, 2)), "variant": int(rng.integers(0, 3))}
+        out.append((case, int(rng.integers(1, 5)), opts))
+    return out
+
+
+@pytest.mark.parametrize("case,path,opts", forced_sample(31, 160),
+                         ids=lambda v: "x".join(map(str, v[1:])) if isinstance(v, tuple) else (str(v) if isinstance(v, int) else "o"))
+def test_random_shape_on_a_forced_family_with_random_options(case, path, opts):
+    """Every family forced in turn (shapes it does not serve are skipped) with the development options toggled at
+    random: fused log-det calls and the flow-step calls against the oracle."""
+    import torch
+    from paper_2410_14634_b200 import binding
+    from oracle import api as oracle, flow_step
+    seed, B, C, H, W, k = case
+    rng = np.random.default_rng(seed)
+    w, y, gx = workloads.make_custom(seed, B, C, H, W, k, sigma=0.05 / np.sqrt(C))
+    s = (rng.uniform(0.5, 1.5, size=C) * rng.choice([-1.0, 1.0], size=C)).astype(np.float32)
+    b = rng.normal(0.0, 0.3, size=C).astype(np.float32)
+    V = (np.linalg.qr(rng.normal(size=(C, C)))[0] + 0.1 * rng.normal(size=(C, C))).astype(np.float32)
+    gl = np.float32(rng.normal())
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+    settings = [(binding.OPT_WARP_RING, opts["ring"], 1), (binding.OPT_WARP_CHANNEL_SPLIT, opts["split"], 1),
+                (binding.OPT_GRADW_TENSOR_PIPE, opts["pipe"], 1), (binding.OPT_DEPENDENT_LAUNCH, opts["pdl"], 1),
+                (binding.OPT_GRADW_SEPARATE, opts["separate"], -1), (binding.OPT_TEAM_VARIANT, opts["variant"], 0)]
+    binding.invconv_set_path(path)
+    for o, v, _ in settings:
+        binding.invconv_set_option(o, v)
+    try:
+        wd, yd, gxd = dev(w), dev(y), dev(gx)
+        x, ld = binding.invconv_forward_logdet(yd, wd)
+        gy, gw = binding.invconv_backward_logdet(gxd, x, wd, torch.tensor([gl], device="cuda"))
+        x2, u, ld2 = binding.invconv_flow_step_forward(yd, wd, dev(s), dev(b), dev(V))
+        gy2, gw2, gs, gb, gV = binding.invconv_flow_step_backward(gxd, x2, wd, dev(s), dev(b), dev(V))
+        torch.cuda.synchronize()
+        status = binding.invconv_get_status()
+    except binding.InvConvError as e:
+        if e.status == binding.UNSUPPORTED:
+            pytest.skip("this family does not serve the shape")
+        raise
+    finally:
+        binding.invconv_set_path(binding.PATH_AUTO)
+        for o, _, default in settings:
+            binding.invconv_set_option(o, default)
+    assert status == 0
+    x_ref = oracle.invconv_forward(y, w)
+    gy_ref, gw_ref = oracle.invconv_backward(gx, x_ref, w)
+    ld_ref = oracle.logdet(w, H, W)
+    assert nmax_err(x.cpu().numpy(), x_ref) <= 1e-4 and nmax_err(gy.cpu().numpy(), gy_ref) <= 1e-4
+    assert nmax_err(gw.cpu().numpy(), gw_ref + gl * oracle.logdet_grad_w(w, H, W)) <= 1e-3
+    assert abs(float(ld.item()) - ld_ref) <= 1e-5 * max(abs(ld_ref), H * W * 1e-3)
+    x_r, u_ref, ldf_ref = flow_step.step_forward(y, w, s, b, V)
+    gy_r, gw_r, gs_ref, gb_ref, gV_ref = flow_step.step_backward(gx, x_r, w, s, b, V)
+    assert nmax_err(u.cpu().numpy(), u_ref) <= 1e-4 and nmax_err(gy2.cpu().numpy(), gy_r) <= 1e-4
+    assert nmax_err(gw2.cpu().numpy(), gw_r) <= 1e-3
+    assert abs(float(ld2.item()) - ldf_ref) <= 1e-5 * max(abs(ldf_ref), H * W * 1e-3)
+    # single-entry sums at one channel can cancel to a thousandth of their terms; the fp32 error of x then shows
+    tol = 1e-4 if C > 1 else 1e-3
+    assert nmax_err(gs.cpu().numpy(), gs_ref) <= tol and nmax_err(gb.cpu().numpy(), gb_ref) <= tol
+    assert nmax_err(gV.cpu().numpy(), gV_ref) <= tol
